@@ -1,0 +1,342 @@
+"""Pins for the CPU oracle: each test ties one part of it to something other than itself
+(the vanilla definition, a closed form printed in the paper, brute force, an invariant)."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import hack_oracle as ho
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand_qkv(rng, b, H, sides, D):
+    qs, ks, vs = [], [], []
+    for s in sides:
+        n = s * s
+        qs.append(rng.standard_normal((b, H, n, D)))
+        ks.append(rng.standard_normal((b, H, n, D)))
+        vs.append(rng.standard_normal((b, H, n, D)))
+    return qs, ks, vs
+
+
+def _run(oracle, qs, ks, vs, layer=0):
+    outs, recs = [], []
+    for k in range(len(qs)):
+        o, r = oracle.scale_step(layer, k, qs[k], ks[k], vs[k])
+        outs.append(o)
+        recs.append(r)
+    return outs, recs
+
+
+# ------------------------------------------------------------------ P1: full budget == vanilla
+def test_full_budget_reproduces_vanilla_attention():
+    """With B_C = B_S >= T_K nothing is ever evicted, so every scale's output must equal
+    uncompressed next-scale attention over all scales <= k (Eq. 3-4)."""
+    rng = np.random.default_rng(1)
+    sides, b, H, D = (1, 2, 3, 4, 5), 2, 3, 8
+    qs, ks, vs = _rand_qkv(rng, b, H, sides, D)
+    T = sum(s * s for s in sides)
+    mask = np.array([[1, 0, 1]])
+    orc = ho.HackOracle(1, H, b, D, sides, mask, budget_c=T, budget_s=T)
+    outs, recs = _run(orc, qs, ks, vs)
+    for bb in range(b):
+        for h in range(H):
+            ref = ho.vanilla_var_attention([q[bb, h] for q in qs], [k[bb, h] for k in ks],
+                                           [v[bb, h] for v in vs], 1.0 / math.sqrt(D))
+            for k in range(len(sides)):
+                np.testing.assert_allclose(outs[k][bb, h], ref[k], rtol=1e-12, atol=1e-13)
+                assert not recs[k][(bb, h)].compressed
+    assert orc.counters.score_pairs == 0
+
+
+def test_trigger_is_strict():
+    """Compression starts only when the candidate count EXCEEDS the budget (T' > B)."""
+    rng = np.random.default_rng(2)
+    sides, D = (1, 2, 3), 4                      # T = 1, 5, 14
+    qs, ks, vs = _rand_qkv(rng, 1, 1, sides, D)
+    orc = ho.HackOracle(1, 1, 1, D, sides, np.array([[1]]), budget_c=5, budget_s=5)
+    _, recs = _run(orc, qs, ks, vs)
+    assert [r[(0, 0)].compressed for r in recs] == [False, False, True]
+    assert [len(r[(0, 0)].keep) for r in recs] == [1, 5, 5]
+
+
+# ------------------------------------------------------------------ P2: softmax rows sum to one
+def test_scores_sum_to_number_of_observation_rows():
+    rng = np.random.default_rng(3)
+    for n_obs, t in [(1, 7), (5, 33), (32, 500)]:
+        q = rng.standard_normal((n_obs, 16)) * 3
+        k = rng.standard_normal((t, 16)) * 3
+        s = ho.subset_attention_scores(q, k, 0.25)
+        assert s.shape == (t,)
+        assert np.all(s >= 0)
+        assert abs(s.sum() - n_obs) < 1e-10
+
+
+def test_scores_match_elementwise_definition():
+    """s_j = sum_i exp(z_ij) / sum_j' exp(z_ij') written out with scalar loops."""
+    rng = np.random.default_rng(4)
+    q = rng.standard_normal((3, 5))
+    k = rng.standard_normal((6, 5))
+    sm = 0.7
+    s = ho.subset_attention_scores(q, k, sm)
+    ref = np.zeros(6)
+    for i in range(3):
+        z = [sm * sum(q[i, d] * k[j, d] for d in range(5)) for j in range(6)]
+        den = sum(math.exp(x) for x in z)
+        for j in range(6):
+            ref[j] += math.exp(z[j]) / den
+    np.testing.assert_allclose(s, ref, rtol=1e-12)
+
+
+def test_observation_rows_uniform_and_complete():
+    assert list(ho.observation_rows(4, 32)) == [0, 1, 2, 3]          # all queries when N_k <= N_obs
+    assert list(ho.observation_rows(64, 32)) == list(range(0, 64, 2))
+    r = ho.observation_rows(100, 32)
+    assert len(r) == 32 and r[0] == 0 and len(set(r)) == 32 and np.all(np.diff(r) >= 3)
+    assert r[-1] < 100
+
+
+# ------------------------------------------------------------------ P3: brute-force selection
+def _best_subset_exhaustive(s, n):
+    """argmax-n subset by exhaustive enumeration; among equal sums the lexicographically
+    smallest index tuple wins (= ties go to lower indices)."""
+    best, best_sum = None, -1.0
+    for comb in itertools.combinations(range(len(s)), n):
+        tot = sum(s[list(comb)])
+        if tot > best_sum + 1e-15:
+            best, best_sum = comb, tot
+    return np.array(best, dtype=np.int64)
+
+
+def test_contextual_selection_is_argmax_subset():
+    rng = np.random.default_rng(5)
+    for t, n in [(6, 2), (8, 3), (9, 8), (10, 1)]:
+        s = rng.random(t)
+        np.testing.assert_array_equal(ho.select_contextual(s, n), _best_subset_exhaustive(s, n))
+
+
+def test_contextual_selection_matches_sort_definition():
+    rng = np.random.default_rng(6)
+    s = np.round(rng.random(200), 2)             # many ties
+    for n in (1, 17, 100, 199, 200, 500):
+        keep = ho.select_contextual(s, n)
+        ranked = sorted(range(200), key=lambda j: (-s[j], j))[: min(n, 200)]
+        np.testing.assert_array_equal(keep, np.array(sorted(ranked)))
+
+
+def test_all_scores_tie_keeps_lowest_indices():
+    """Constant queries make every logit equal, so all scores tie and the lowest indices win."""
+    k = np.random.default_rng(7).standard_normal((40, 8))
+    q = np.zeros((32, 8))
+    s = ho.subset_attention_scores(q, k, 0.3)
+    np.testing.assert_allclose(s, 32 / 40)
+    np.testing.assert_array_equal(ho.select_contextual(s, 11), np.arange(11))
+
+
+# ------------------------------------------------------------------ P4/P5/P10: structural rule
+def test_structural_keeps_initial_and_latest_scales():
+    rng = np.random.default_rng(8)
+    sides, D = (1, 2, 3, 4, 5, 6), 8            # N = 1,4,9,16,25,36 ; T = 1,5,14,30,55,91
+    qs, ks, vs = _rand_qkv(rng, 1, 2, sides, D)
+    mask = np.array([[0, 1]])
+    b_s, b_c = 50, 12
+    orc = ho.HackOracle(1, 2, 1, D, sides, mask, budget_c=b_c, budget_s=b_s)
+    starts = np.concatenate([[0], np.cumsum([s * s for s in sides])])
+    seen_evicted = [set(), set()]
+    prev_pos = [np.zeros(0, np.int64)] * 2
+    for k in range(len(sides)):
+        n_k = sides[k] ** 2
+        _, recs = orc.scale_step(0, k, qs[k], ks[k], vs[k])
+        for h in (0, 1):
+            pos = recs[(0, h)].pos
+            assert np.all(np.diff(pos) > 0)                          # ascending, unique
+            cand = set(prev_pos[h].tolist()) | set(range(starts[k], starts[k + 1]))
+            assert set(pos.tolist()) <= cand                         # only candidates survive
+            assert not (set(pos.tolist()) & seen_evicted[h])         # evicted never returns
+            seen_evicted[h] |= cand - set(pos.tolist())
+            prev_pos[h] = pos
+        pos_s = set(recs[(0, 0)].pos.tolist())
+        assert set(range(0, min(5, starts[k + 1]))) <= pos_s         # scales 1-2 (5 tokens)
+        assert set(range(starts[k], starts[k + 1])) <= pos_s         # latest scale
+        t_cand = recs[(0, 0)].n_candidates
+        n_prot = min(5, starts[k + 1]) + (n_k if k >= 2 else 0)
+        assert len(pos_s) == min(t_cand, max(b_s, n_prot))
+        assert len(recs[(0, 1)].pos) == min(recs[(0, 1)].n_candidates, b_c)
+    assert orc.counters.overflows == 0
+
+
+def test_structural_zero_free_budget_keeps_exactly_protected():
+    """B_S = N_init + N_k  (M = 0)  =>  kept = first two scales + current scale, nothing else."""
+    s = np.random.default_rng(9).random(5 + 9 + 16)
+    sid = np.array([1] + [2] * 4 + [3] * 9 + [4] * 16)
+    keep = ho.select_structural(s, sid, 4, 2, 5 + 16)
+    np.testing.assert_array_equal(keep, np.concatenate([np.arange(5), np.arange(14, 30)]))
+
+
+def test_structural_free_slots_filled_by_score():
+    s = np.array([9, 9, 9, 9, 9, .1, .5, .3, .5, .2, 9, 9, 9], dtype=float)
+    sid = np.array([1, 2, 2, 2, 2, 3, 3, 3, 3, 3, 4, 4, 4])
+    keep = ho.select_structural(s, sid, 4, 2, 5 + 3 + 2)
+    np.testing.assert_array_equal(keep, [0, 1, 2, 3, 4, 6, 8, 10, 11, 12])   # ties -> lower index
+    keep = ho.select_structural(s, sid, 4, 2, 5 + 3 + 3)
+    np.testing.assert_array_equal(keep, [0, 1, 2, 3, 4, 6, 7, 8, 10, 11, 12])
+
+
+def test_structural_overflow_policies():
+    """B_S smaller than the protected set: policy 0 keeps all protected entries (more than B_S),
+    policy 1 lets the current scale compete and keeps exactly B_S."""
+    rng = np.random.default_rng(10)
+    s = rng.random(5 + 9 + 16)
+    sid = np.array([1] + [2] * 4 + [3] * 9 + [4] * 16)
+    keep0 = ho.select_structural(s, sid, 4, 2, 12, ho.KEEP_PROTECTED)
+    np.testing.assert_array_equal(keep0, np.concatenate([np.arange(5), np.arange(14, 30)]))
+    keep1 = ho.select_structural(s, sid, 4, 2, 12, ho.COMPETE)
+    assert len(keep1) == 12 and set(range(5)) <= set(keep1.tolist())
+    rest = np.array(sorted(set(keep1.tolist()) - set(range(5))))
+    ranked = sorted(range(5, 30), key=lambda j: (-s[j], j))[:7]
+    np.testing.assert_array_equal(rest, sorted(ranked))
+
+
+# ------------------------------------------------------------------ P6: compaction copies rows
+def test_stored_rows_are_bit_copies_of_inputs():
+    rng = np.random.default_rng(11)
+    sides, D = (1, 2, 3, 4, 5), 4
+    qs, ks, vs = _rand_qkv(rng, 1, 2, sides, D)
+    orc = ho.HackOracle(1, 2, 1, D, sides, np.array([[1, 0]]), budget_c=9, budget_s=30)
+    _run(orc, qs, ks, vs)
+    k_all = np.concatenate([k[0] for k in ks], axis=1)
+    v_all = np.concatenate([v[0] for v in vs], axis=1)
+    for h in range(2):
+        st = orc.state[0][0][h]
+        assert np.array_equal(st.k, k_all[h][st.pos])
+        assert np.array_equal(st.v, v_all[h][st.pos])
+        assert np.all(np.diff(st.pos) > 0)
+    assert orc.state[0][0][0].k.shape[0] == 9
+
+
+# ------------------------------------------------------------------ P7: attention properties
+def test_attention_is_convex_combination_and_permutation_invariant():
+    rng = np.random.default_rng(12)
+    q = rng.standard_normal((7, 8)) * 2
+    k = rng.standard_normal((19, 8))
+    v = rng.standard_normal((19, 8))
+    o = ho.attend(q, k, v, 0.35)
+    assert np.all(o <= v.max(axis=0) + 1e-12) and np.all(o >= v.min(axis=0) - 1e-12)
+    perm = rng.permutation(19)
+    np.testing.assert_allclose(ho.attend(q, k[perm], v[perm], 0.35), o, rtol=1e-12, atol=1e-14)
+    # one key only -> output is that key's value; identical keys -> mean of values
+    np.testing.assert_allclose(ho.attend(q, k[:1], v[:1], 0.35), np.repeat(v[:1], 7, axis=0))
+    np.testing.assert_allclose(ho.attend(q, np.repeat(k[:1], 19, axis=0), v, 0.35),
+                               np.repeat(v.mean(axis=0, keepdims=True), 7, axis=0), rtol=1e-12)
+
+
+def test_attention_scale_and_transpose_sensitivity():
+    """A dominant logit pins the output to one value row: catches a dropped sm_scale, a
+    transposed operand or a sign error."""
+    D = 4
+    k = np.eye(D)[:3] * 50.0                      # three orthogonal keys
+    v = np.array([[1., 0, 0, 0], [0, 2., 0, 0], [0, 0, 3., 0]])
+    q = np.array([[0, 1., 0, 0]])                 # matches key 1
+    o = ho.attend(q, k, v, 1.0)
+    np.testing.assert_allclose(o, v[1:2], atol=1e-12)
+    o_small = ho.attend(q, k, v, 1e-9)            # scale -> 0 gives the plain mean
+    np.testing.assert_allclose(o_small, v.mean(axis=0, keepdims=True), atol=1e-6)
+
+
+# ------------------------------------------------------------------ P8: complexity closed forms
+def _golden_rows(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(line.split())
+    return rows
+
+
+@pytest.mark.parametrize("row", _golden_rows("complexity_closed_forms.txt"))
+def test_counters_match_closed_forms(row):
+    a, K, t_final, total_pairs = (int(x) for x in row)
+    sides = tuple(a ** k for k in range(K))
+    D = 2
+    rng = np.random.default_rng(13)
+    qs, ks, vs = _rand_qkv(rng, 1, 1, sides, D)
+    # full cache: attention pairs = sum N_k T_k  (Eq. 15-17), T_K = Eq. 14
+    T = sum(s * s for s in sides)
+    assert T == t_final == (a ** (2 * K) - 1) // (a * a - 1)
+    orc = ho.HackOracle(1, 1, 1, D, sides, np.array([[1]]), budget_c=T, budget_s=T)
+    _run(orc, qs, ks, vs)
+    assert orc.counters.attention_pairs == total_pairs
+    num = 1 - a ** (2 * K) - a ** (2 * K + 2) + a ** (4 * K + 2)
+    den = (a * a - 1) ** 2 * (a * a + 1)
+    assert num % den == 0 and num // den == total_pairs
+    # budgeted: pairs = sum N_k min(T_k, B) <= B sum N_k (Eq. 12 / 18-21); overhead bound Eq. 13 / 22
+    for B in (3, 7, max(T // 3, 1)):
+        orc = ho.HackOracle(1, 1, 1, D, sides, np.array([[1]]), budget_c=B, budget_s=B, n_obs=4)
+        _run(orc, qs, ks, vs)
+        n = [s * s for s in sides]
+        t_k = np.cumsum(n)
+        assert orc.counters.attention_pairs == sum(nk * min(tk, B) for nk, tk in zip(n, t_k))
+        assert orc.counters.attention_pairs <= B * sum(n)
+        k_s = next((i for i, tk in enumerate(t_k) if tk > B), None)
+        if k_s is not None:
+            assert orc.counters.score_pairs <= sum(4 * (B + nk) for nk in n[k_s:])
+            assert orc.counters.score_pairs > 0
+
+
+# ------------------------------------------------------------------ P9: f_C against a 10-line brute force
+def test_contextual_step_equals_full_column_sum_topk():
+    """All heads contextual and N_obs >= N_k: the kept set is the top-B of the column sums of the
+    FULL attention matrix of the step, computed here from scratch."""
+    rng = np.random.default_rng(14)
+    sides, D, B = (1, 2, 3, 4), 6, 11
+    qs, ks, vs = _rand_qkv(rng, 1, 1, sides, D)
+    orc = ho.HackOracle(1, 1, 1, D, sides, np.array([[1]]), budget_c=B, budget_s=B, n_obs=64)
+    kept_pos = np.zeros(0, dtype=np.int64)
+    k_all = np.concatenate([k[0, 0] for k in ks])
+    start = 0
+    for k in range(len(sides)):
+        n_k = sides[k] ** 2
+        cand = np.concatenate([kept_pos, np.arange(start, start + n_k)])
+        start += n_k
+        if len(cand) > B:
+            logits = (qs[k][0, 0] @ k_all[cand].T) / math.sqrt(D)
+            A = np.exp(logits - logits.max(1, keepdims=True))
+            A /= A.sum(1, keepdims=True)
+            col = A.sum(0)
+            kept_pos = np.sort(cand[sorted(range(len(cand)), key=lambda j: (-col[j], j))[:B]])
+        else:
+            kept_pos = cand
+        _, recs = orc.scale_step(0, k, qs[k], ks[k], vs[k])
+        np.testing.assert_array_equal(recs[(0, 0)].pos, kept_pos)
+
+
+# ------------------------------------------------------------------ budgets (Eq. 7)
+@pytest.mark.parametrize("row", _golden_rows("budgets.txt"))
+def test_budget_split_matches_hand_derivation(row):
+    t_k, frac, alpha, rule, param = int(row[0]), float(row[1]), float(row[2]), row[3], float(row[4])
+    b, b_c, b_s = int(row[5]), int(row[6]), int(row[7])
+    assert int(math.floor(frac * t_k + 1e-9)) == b
+    assert ho.split_budget(b, alpha, rule, param, t_k) == (b_c, b_s)
+    if b_s < t_k:
+        assert alpha * b_c + (1 - alpha) * b_s <= b + 1e-9           # Eq. 7 as an upper bound
+
+
+def test_mean_kept_length_within_budget():
+    """No overflow => the stack-mean kept length never exceeds B (Eq. 7)."""
+    rng = np.random.default_rng(15)
+    sides, D, H = (1, 2, 3, 4, 5, 6, 7), 4, 4       # T_K = 140
+    T = sum(s * s for s in sides)
+    B = int(0.5 * T)
+    alpha = 0.5
+    b_c, b_s = ho.split_budget(B, alpha, "fraction", 0.1, T)
+    qs, ks, vs = _rand_qkv(rng, 1, H, sides, D)
+    orc = ho.HackOracle(1, H, 1, D, sides, np.array([[1, 0, 1, 0]]), budget_c=b_c, budget_s=b_s)
+    for k in range(len(sides)):
+        orc.scale_step(0, k, qs[k], ks[k], vs[k])
+        assert orc.stored_lengths(0).mean() <= B
+    assert orc.counters.overflows == 0
+    assert orc.counters.peak_entries == orc.stored_lengths(0).sum()

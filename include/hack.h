@@ -1,0 +1,183 @@
+/*
+ * hack.h - C ABI of the B200 (sm_100a) library for the per-scale decoding step of head-aware
+ * KV-cache compression in next-scale visual autoregressive transformers.
+ *
+ * One "step" serves one (layer, scale): the new scale's keys/values join the cache (Eq. 3), every
+ * candidate key of a head whose cache would exceed its budget is scored with a small query subset
+ * (Eq. 9), a budgeted subset is selected per head with the contextual rule (Eq. 10) or the
+ * structural rule (Eq. 11) under asymmetric budgets (Eq. 7-8), the survivors are compacted into a
+ * ragged per-head cache, and the scale's queries attend over it (Eq. 4 on the compressed cache,
+ * compression preceding attention, section "Asymmetric Head Budget Allocation").
+ *
+ * Conventions for every entry point
+ *  - Q, K, V, O are CALLER-OWNED DEVICE buffers, dense row-major [batch, n_heads, N_k, head_dim]
+ *    in the cache's dtype, 16-byte aligned, N_k = side_k^2 of the scale being decoded.  Only the
+ *    *_host entry point takes host pointers.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only
+ *    enqueue work and return; nothing synchronises unless stated.
+ *  - Layers and scales are 0-based.  Each layer walks its scales in order 0,1,2,...; a call for
+ *    any other scale returns HACK_ERR_STATE.  Within a scale a layer is served either by
+ *    hack_scale_step, or by [hack_score, hack_select,] hack_compact, hack_attend in that order.
+ *  - Stored lengths are a function of the schedule, the budgets and the head type only (the
+ *    selection decides WHICH entries survive, never HOW MANY), so the library keeps them on the
+ *    host and never reads anything back from the device to plan a launch.
+ *  - Candidate index j of a head in a step: j < L addresses the L entries stored before the step
+ *    (ascending original position), j >= L the new scale's token j - L.
+ *  - Argument errors are detected on the host before anything is launched and leave the cache
+ *    unchanged.  Nothing traps on the device.  There is no CPU fallback.
+ *  - The cache (K/V planes, position plane, scratch) is owned by the library and released by
+ *    hack_free_cache.  A cache is not thread safe; use one cache per stream of work.
+ */
+#ifndef HACK_H_
+#define HACK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define HACK_API __attribute__((visibility("default")))
+#else
+#define HACK_API
+#endif
+
+typedef struct hack_cache hack_cache_t; /* opaque, library-owned */
+
+typedef enum {
+  HACK_OK = 0,
+  HACK_ERR_INVALID_ARG = 1, /* NULL pointer, size or index out of range, misaligned buffer */
+  HACK_ERR_UNSUPPORTED = 2, /* head_dim / dtype / n_obs outside what the kernels implement */
+  HACK_ERR_OOM = 3,         /* device or host allocation failed */
+  HACK_ERR_CUDA = 4,        /* a CUDA call failed; hack_last_error() has the text */
+  HACK_ERR_STATE = 5,       /* call out of order for this layer (wrong scale or phase) */
+  HACK_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by hack_poll_status) */
+} hack_status_t;
+
+typedef enum { HACK_F32 = 0, HACK_BF16 = 1 } hack_dtype_t;
+
+/* Overflow rule for structural heads when B_S < N_init + N_k (the paper is silent): */
+enum { HACK_OVERFLOW_KEEP_PROTECTED = 0, /* keep every protected entry, exceed B_S */
+       HACK_OVERFLOW_COMPETE = 1 };      /* protect only the initial scales; keep exactly B_S */
+
+typedef struct {
+  int32_t n_layers, n_heads, head_dim, batch; /* head_dim in {64, 128} */
+  int32_t n_scales;
+  const int32_t* scale_sides;        /* host, [n_scales], copied at init; N_k = side^2 */
+  int32_t dtype;                     /* hack_dtype_t of Q/K/V/O and of the cache */
+  const uint8_t* head_is_contextual; /* host, [n_layers*n_heads], 1 = contextual, 0 = structural
+                                        (offline classification, Eq. 6); copied at init */
+  int32_t budget_c, budget_s;        /* B_C, B_S: entries per head, >= 1 (Eq. 7-8) */
+  int32_t n_obs;                     /* query subset size N_obs, 1..32 (Eq. 9; paper uses 32) */
+  int32_t n_init_scales;             /* leading scales always kept in structural heads (paper: 2) */
+  float sm_scale;                    /* softmax scale; 0 selects 1/sqrt(head_dim) */
+  int32_t overflow_policy;           /* HACK_OVERFLOW_* */
+  int32_t device;                    /* CUDA device ordinal */
+} hack_config_t;
+
+/* Host-side plan of one step of one layer (all lengths in entries per head). */
+typedef struct {
+  int32_t n_new;                 /* N_k */
+  int32_t stored_c, stored_s;    /* L before the step, contextual / structural heads */
+  int32_t cand_c, cand_s;        /* T' = L + N_k */
+  int32_t kept_c, kept_s;        /* length after the step */
+  int32_t triggered_c, triggered_s; /* 1 if T' exceeds the type's budget (strictly) */
+  int32_t n_obs_rows;            /* min(N_obs, N_k) */
+} hack_step_info_t;
+
+/* Buffer strides a caller of the separate stage calls must use. */
+typedef struct {
+  int32_t cand_stride; /* floats per (batch, head) row of `scores`: max T' over all steps */
+  int32_t kept_stride; /* int32 per (batch, head) row of `idx`: max kept length over all steps */
+  int32_t max_new;     /* largest N_k */
+} hack_limits_t;
+
+/* Eq. 7, B = alpha*B_C + (1-alpha)*B_S, solved under one of the paper's two allocation rules
+ * (appendix, "Model-Specific Configurations").  Host only, no device work.
+ *   rule 0 ("fraction"): B_C = floor(param*T_K); B_S = floor((B - alpha*B_C)/(1-alpha)).
+ *   rule 1 ("ratio"):    B_C : B_S = 1 : param; B_C = floor(B/(alpha+param*(1-alpha))), B_S = param*B_C.
+ * B_S is clamped to T_K and both results are at least 1.  INVALID_ARG unless 0 < alpha < 1. */
+HACK_API hack_status_t hack_split_budget(int32_t budget, double alpha, int32_t rule, double param,
+                                int32_t total_tokens, int32_t* budget_c, int32_t* budget_s);
+
+/* Allocate the ragged per-head cache for the whole stack (Eq. 5, 8: per head at most its type's
+ * budget, or the protected set if that is larger) and all scratch.  *out is set only on
+ * success.  Capacity per head = the largest stored length its type reaches over the schedule. */
+HACK_API hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out);
+/* Release everything; synchronises the device first.  NULL is accepted. */
+HACK_API hack_status_t hack_free_cache(hack_cache_t* cache);
+/* New image: all layers back to scale 0 with empty caches.  Enqueues nothing. */
+HACK_API hack_status_t hack_reset(hack_cache_t* cache);
+
+HACK_API hack_status_t hack_get_limits(const hack_cache_t* cache, hack_limits_t* out);
+/* Plan of step (layer, scale) given the layer's current state; scale must be the layer's next. */
+HACK_API hack_status_t hack_step_info(const hack_cache_t* cache, int32_t layer, int32_t scale,
+                             hack_step_info_t* out);
+
+/* Subset-attention importance (Eq. 9 and the TOPK argument of Eq. 10-11).  For every (b,h) whose
+ * type is triggered in this step: scores[(b*H+h)*cand_stride + j] = sum over the
+ * min(N_obs, N_k) uniformly spaced query rows i = floor(m*N_k/n) of
+ * Softmax_j(sm_scale * <Q[i], K_cand[j]>) over all T' candidates (stored ++ k_new).  Rows of
+ * heads that are not triggered are left untouched.  Does not change the cache. */
+HACK_API hack_status_t hack_score(hack_cache_t* cache, int32_t layer, int32_t scale, const void* q,
+                         const void* k_new, float* scores, void* stream);
+
+/* Budgeted selection per head from fp32 `scores` (layout as above).  Contextual heads keep the
+ * B_C best candidates (Eq. 10).  Structural heads keep every entry of the first n_init_scales
+ * scales and of the scale being decoded and fill the remaining M = B_S - |protected| slots with
+ * the best of the rest (Eq. 11).  Order: score descending on the fp32 bit pattern, ties to the
+ * lower candidate index.  Heads that are not triggered keep everything.  Output
+ * idx[(b*H+h)*kept_stride + r], r < kept, ascending candidate indices; kept_out[b*H+h] their
+ * count (may be NULL).  Does not change the cache. */
+HACK_API hack_status_t hack_select(hack_cache_t* cache, int32_t layer, int32_t scale, const float* scores,
+                          int32_t* idx, int32_t* kept_out, void* stream);
+
+/* Gather the surviving K/V rows (Eq. 10-11) into the layer's ragged cache in ascending original
+ * position; evicted entries are gone for good.  `idx` as written by hack_select for this step;
+ * each head's row must hold exactly hack_step_info's kept_c / kept_s entries.  In place. */
+HACK_API hack_status_t hack_compact(hack_cache_t* cache, int32_t layer, int32_t scale, const int32_t* idx,
+                           const void* k_new, const void* v_new, void* stream);
+
+/* O = Softmax(sm_scale * Q K^T) V over the head's compacted cache, all N_k queries, no mask
+ * inside the scale (Eq. 4 on the compressed cache).  Requires hack_compact for this scale;
+ * completes the step (the layer then expects scale + 1). */
+HACK_API hack_status_t hack_attend(hack_cache_t* cache, int32_t layer, int32_t scale, const void* q,
+                          void* out, void* stream);
+
+/* The whole step for one (layer, scale): score -> select -> compact -> attend; heads whose
+ * candidate count does not exceed their budget skip scoring and selection and keep everything
+ * (section "KV Cache Compression for VAR": compress whenever the length exceeds the budget). */
+HACK_API hack_status_t hack_scale_step(hack_cache_t* cache, int32_t layer, int32_t scale, const void* q,
+                              const void* k, const void* v, void* out, void* stream);
+
+/* Same step with HOST buffers (pinned memory recommended): copies Q/K/V to library-owned device
+ * staging, runs the step, copies O back, all on `stream`, and returns without synchronising.
+ * The staging buffers are allocated by the first such call on a cache. */
+HACK_API hack_status_t hack_scale_step_host(hack_cache_t* cache, int32_t layer, int32_t scale,
+                                   const void* q_host, const void* k_host, const void* v_host,
+                                   void* out_host, void* stream);
+
+/* Stored length of every (batch, head) of a layer, host_out[b*H+h].  Host bookkeeping only. */
+HACK_API hack_status_t hack_get_lengths(const hack_cache_t* cache, int32_t layer, int32_t* host_out);
+/* Test inspection (synchronises the device): copy one head's stored rows to host memory.
+ * which = 0: K rows, 1: V rows (dtype of the cache, [len, head_dim]); 2: original global token
+ * positions (int32 [len]).  `bytes` is the size of host_out and must cover the stored length. */
+HACK_API hack_status_t hack_read_head(hack_cache_t* cache, int32_t layer, int32_t b, int32_t h,
+                             int32_t which, void* host_out, size_t bytes);
+
+/* KV bytes (K and V rows only): currently stored, the peak since init/reset, and reserved. */
+HACK_API hack_status_t hack_kv_bytes(const hack_cache_t* cache, size_t* live, size_t* peak, size_t* reserved);
+/* Number of the library's own kernel launches enqueued through this cache since init. */
+HACK_API hack_status_t hack_launch_count(const hack_cache_t* cache, uint64_t* launches);
+/* Synchronises `stream`, then reports the device status word: HACK_OK, or HACK_ERR_TIMEOUT if a
+ * bounded device-side wait gave up (the word is cleared by the call). */
+HACK_API hack_status_t hack_poll_status(hack_cache_t* cache, void* stream);
+/* Text of the calling thread's last error; never NULL. */
+HACK_API const char* hack_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HACK_H_ */

@@ -1,0 +1,526 @@
+// Host side of the C ABI: argument checks, the per-layer state machine, the deterministic length
+// plan of every step, cache and scratch allocation, and the launch sequence of the step.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "hack_internal.h"
+
+namespace hack {
+
+static thread_local std::string g_last_error;
+void set_error(const std::string& msg) { g_last_error = msg; }
+
+int launch_attend_simt(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st);
+
+int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st) {
+  return launch_attend_simt(a, dtype, q, out, st);
+}
+
+}  // namespace hack
+
+using hack::set_error;
+
+struct LayerState {
+  int next_scale = 0;
+  int phase = 0;          // 0: scale not started; 1: compacted, attention pending
+  int len[2] = {0, 0};    // stored length per head type ([0] structural, [1] contextual)
+};
+
+struct hack_cache {
+  hack_config_t cfg;
+  std::vector<int32_t> sides, n_tok, t_cum;     // t_cum[k] = tokens of scales 0..k
+  std::vector<uint8_t> mask;                    // host copy [L*H]
+  int elt = 2;
+  int budget[2] = {0, 0};
+  int cap[2] = {0, 0};
+  int t_init = 0;
+  float sm_scale = 0.f;
+  hack_limits_t limits{};
+  std::vector<LayerState> layers;
+  std::vector<size_t> layer_rows;               // rows per plane of each layer
+  std::vector<size_t> layer_row_base;           // first row of each layer inside the big planes
+  std::vector<int> n_ctx_heads;                 // contextual heads per layer
+  // device memory
+  unsigned char* k_all = nullptr;
+  unsigned char* v_all = nullptr;
+  int32_t* pos_all = nullptr;
+  int32_t* row_off = nullptr;                   // [L][b*H]
+  std::vector<int32_t> row_off_host;            // same table on the host
+  uint8_t* mask_dev = nullptr;                  // [L*H]
+  float* scores = nullptr;                      // [b*H, cand_stride]
+  int32_t* idx = nullptr;                       // [b*H, kept_stride]
+  hack::Scratch scratch{};
+  int* status = nullptr;
+  unsigned char* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging
+  size_t reserved_bytes = 0, peak_bytes = 0;
+  uint64_t launches = 0;
+};
+
+namespace {
+
+#define HACK_CUDA(call)                                                              \
+  do {                                                                               \
+    cudaError_t e_ = (call);                                                         \
+    if (e_ != cudaSuccess) {                                                         \
+      set_error(std::string(#call) + ": " + cudaGetErrorString(e_));                 \
+      return e_ == cudaErrorMemoryAllocation ? HACK_ERR_OOM : HACK_ERR_CUDA;         \
+    }                                                                                \
+  } while (0)
+
+hack_status_t fail(hack_status_t s, const char* msg) {
+  set_error(msg);
+  return s;
+}
+
+// Length plan of one step from the layer's current lengths.  Pure host arithmetic: the stored
+// length after a step depends on the schedule, the budget and the head type only.
+void plan_step(const hack_cache* c, const LayerState& ls, int scale, hack_step_info_t* p) {
+  const int n_new = c->n_tok[scale];
+  p->n_new = n_new;
+  p->n_obs_rows = std::min(c->cfg.n_obs, n_new);
+  int cand[2], kept[2], trig[2];
+  for (int t = 0; t < 2; ++t) {
+    const int L = ls.len[t];
+    cand[t] = L + n_new;
+    if (cand[t] <= c->budget[t]) {            // compress only when the budget is exceeded
+      kept[t] = cand[t];
+      trig[t] = 0;
+    } else {
+      trig[t] = 1;
+      if (t == 1) {
+        kept[t] = c->budget[t];
+      } else {
+        int prot;
+        if (scale < c->cfg.n_init_scales) prot = cand[t];
+        else if (c->cfg.overflow_policy == HACK_OVERFLOW_KEEP_PROTECTED) prot = std::min(L, c->t_init) + n_new;
+        else prot = std::min(L, c->t_init);
+        kept[t] = std::min(cand[t], std::max(c->budget[t], prot));
+      }
+    }
+  }
+  p->stored_s = ls.len[0]; p->stored_c = ls.len[1];
+  p->cand_s = cand[0];     p->cand_c = cand[1];
+  p->kept_s = kept[0];     p->kept_c = kept[1];
+  p->triggered_s = trig[0]; p->triggered_c = trig[1];
+}
+
+hack::StepArgs make_args(const hack_cache* c, int layer, int scale, const hack_step_info_t& p) {
+  hack::StepArgs a{};
+  a.n_heads = c->cfg.n_heads; a.batch = c->cfg.batch; a.head_dim = c->cfg.head_dim;
+  a.n_new = p.n_new;
+  a.stored[0] = p.stored_s; a.stored[1] = p.stored_c;
+  a.cand[0] = p.cand_s;     a.cand[1] = p.cand_c;
+  a.kept[0] = p.kept_s;     a.kept[1] = p.kept_c;
+  a.trig[0] = p.triggered_s; a.trig[1] = p.triggered_c;
+  a.n_obs_rows = p.n_obs_rows;
+  a.sm_scale = c->sm_scale;
+  a.t_init = c->t_init;
+  a.protect_new = (c->cfg.overflow_policy == HACK_OVERFLOW_KEEP_PROTECTED) || scale < c->cfg.n_init_scales;
+  a.pos_base = scale == 0 ? 0 : c->t_cum[scale - 1];
+  a.cand_stride = c->limits.cand_stride;
+  a.kept_stride = c->limits.kept_stride;
+  a.is_ctx = c->mask_dev + (size_t)layer * c->cfg.n_heads;
+  a.row_off = c->row_off + (size_t)layer * c->cfg.batch * c->cfg.n_heads;
+  const size_t row_bytes = (size_t)c->cfg.head_dim * c->elt;
+  a.k_plane = c->k_all + c->layer_row_base[layer] * row_bytes;
+  a.v_plane = c->v_all + c->layer_row_base[layer] * row_bytes;
+  a.pos_plane = c->pos_all + c->layer_row_base[layer];
+  a.status = c->status;
+  return a;
+}
+
+size_t live_bytes(const hack_cache* c) {
+  size_t rows = 0;
+  for (int l = 0; l < c->cfg.n_layers; ++l) {
+    const LayerState& ls = c->layers[l];
+    rows += (size_t)c->cfg.batch * ((size_t)c->n_ctx_heads[l] * ls.len[1] +
+                                    (size_t)(c->cfg.n_heads - c->n_ctx_heads[l]) * ls.len[0]);
+  }
+  return rows * c->cfg.head_dim * c->elt * 2;
+}
+
+hack_status_t check_step(const hack_cache* c, int layer, int scale, int want_phase) {
+  if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
+  if (layer < 0 || layer >= c->cfg.n_layers) return fail(HACK_ERR_INVALID_ARG, "layer out of range");
+  if (scale < 0 || scale >= c->cfg.n_scales) return fail(HACK_ERR_INVALID_ARG, "scale out of range");
+  const LayerState& ls = c->layers[layer];
+  if (scale != ls.next_scale) return fail(HACK_ERR_STATE, "this layer expects a different scale");
+  if (ls.phase != want_phase)
+    return fail(HACK_ERR_STATE, want_phase ? "hack_compact must precede hack_attend for this scale"
+                                           : "this scale is already compacted; call hack_attend");
+  return HACK_OK;
+}
+
+bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+void advance_after_compact(hack_cache* c, int layer, const hack_step_info_t& p) {
+  LayerState& ls = c->layers[layer];
+  ls.len[0] = p.kept_s;
+  ls.len[1] = p.kept_c;
+  ls.phase = 1;
+  c->peak_bytes = std::max(c->peak_bytes, live_bytes(c));
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* hack_last_error(void) { return hack::g_last_error.c_str(); }
+
+hack_status_t hack_split_budget(int32_t budget, double alpha, int32_t rule, double param,
+                                int32_t total_tokens, int32_t* budget_c, int32_t* budget_s) {
+  if (!budget_c || !budget_s) return fail(HACK_ERR_INVALID_ARG, "output pointer is NULL");
+  if (!(alpha > 0.0 && alpha < 1.0)) return fail(HACK_ERR_INVALID_ARG, "alpha must be in (0,1)");
+  if (budget < 1 || total_tokens < 1 || !(param > 0.0)) return fail(HACK_ERR_INVALID_ARG, "budget, total_tokens and param must be positive");
+  const double eps = 1e-9;
+  long long bc, bs;
+  if (rule == 0) {
+    bc = (long long)std::floor(param * total_tokens + eps);
+    bs = (long long)std::floor((budget - alpha * (double)bc) / (1.0 - alpha) + eps);
+  } else if (rule == 1) {
+    bc = (long long)std::floor(budget / (alpha + param * (1.0 - alpha)) + eps);
+    bs = (long long)std::llround(param * (double)bc);
+  } else {
+    return fail(HACK_ERR_INVALID_ARG, "rule must be 0 (fraction) or 1 (ratio)");
+  }
+  bs = std::min<long long>(bs, total_tokens);
+  *budget_c = (int32_t)std::max<long long>(bc, 1);
+  *budget_s = (int32_t)std::max<long long>(bs, 1);
+  return HACK_OK;
+}
+
+hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
+  if (!cfg || !out) return fail(HACK_ERR_INVALID_ARG, "cfg or out is NULL");
+  if (!cfg->scale_sides || !cfg->head_is_contextual) return fail(HACK_ERR_INVALID_ARG, "scale_sides or head_is_contextual is NULL");
+  if (cfg->n_layers < 1 || cfg->n_heads < 1 || cfg->batch < 1 || cfg->n_scales < 1)
+    return fail(HACK_ERR_INVALID_ARG, "n_layers, n_heads, batch and n_scales must be positive");
+  if (cfg->budget_c < 1 || cfg->budget_s < 1) return fail(HACK_ERR_INVALID_ARG, "budgets must be at least 1");
+  if (cfg->n_init_scales < 0 || cfg->n_init_scales > cfg->n_scales) return fail(HACK_ERR_INVALID_ARG, "n_init_scales out of range");
+  if (cfg->overflow_policy != 0 && cfg->overflow_policy != 1) return fail(HACK_ERR_INVALID_ARG, "unknown overflow_policy");
+  if (cfg->sm_scale < 0.f || !std::isfinite(cfg->sm_scale)) return fail(HACK_ERR_INVALID_ARG, "sm_scale must be finite and non-negative");
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return fail(HACK_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+  if (cfg->dtype != HACK_F32 && cfg->dtype != HACK_BF16) return fail(HACK_ERR_UNSUPPORTED, "dtype must be HACK_F32 or HACK_BF16");
+  if (cfg->n_obs < 1 || cfg->n_obs > hack::kMaxObs) return fail(HACK_ERR_UNSUPPORTED, "n_obs must be in 1..32");
+  for (int k = 0; k < cfg->n_scales; ++k)
+    if (cfg->scale_sides[k] < 1 || cfg->scale_sides[k] > 1024) return fail(HACK_ERR_INVALID_ARG, "scale side out of range (1..1024)");
+  for (int i = 0; i < cfg->n_layers * cfg->n_heads; ++i)
+    if (cfg->head_is_contextual[i] > 1) return fail(HACK_ERR_INVALID_ARG, "head_is_contextual must hold 0 or 1");
+  int n_dev = 0;
+  HACK_CUDA(cudaGetDeviceCount(&n_dev));
+  if (cfg->device < 0 || cfg->device >= n_dev) return fail(HACK_ERR_INVALID_ARG, "device ordinal out of range");
+  HACK_CUDA(cudaSetDevice(cfg->device));
+
+  hack_cache* c = new (std::nothrow) hack_cache();
+  if (!c) return fail(HACK_ERR_OOM, "host allocation failed");
+  c->cfg = *cfg;
+  c->sides.assign(cfg->scale_sides, cfg->scale_sides + cfg->n_scales);
+  c->mask.assign(cfg->head_is_contextual, cfg->head_is_contextual + (size_t)cfg->n_layers * cfg->n_heads);
+  c->cfg.scale_sides = c->sides.data();
+  c->cfg.head_is_contextual = c->mask.data();
+  c->elt = cfg->dtype == HACK_F32 ? 4 : 2;
+  c->budget[0] = cfg->budget_s;
+  c->budget[1] = cfg->budget_c;
+  c->sm_scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+  long long cum = 0;
+  for (int k = 0; k < cfg->n_scales; ++k) {
+    c->n_tok.push_back(c->sides[k] * c->sides[k]);
+    cum += c->n_tok[k];
+    if (cum > (1ll << 28)) { delete c; return fail(HACK_ERR_UNSUPPORTED, "schedule too long"); }
+    c->t_cum.push_back((int32_t)cum);
+  }
+  c->t_init = cfg->n_init_scales > 0 ? c->t_cum[cfg->n_init_scales - 1] : 0;
+  // walk the schedule once to find capacities and buffer strides
+  {
+    LayerState ls;
+    int cand_max = 1, kept_max = 1, new_max = 1;
+    for (int k = 0; k < cfg->n_scales; ++k) {
+      hack_step_info_t p;
+      plan_step(c, ls, k, &p);
+      cand_max = std::max({cand_max, p.cand_c, p.cand_s});
+      kept_max = std::max({kept_max, p.kept_c, p.kept_s});
+      new_max = std::max(new_max, p.n_new);
+      c->cap[0] = std::max(c->cap[0], p.kept_s);
+      c->cap[1] = std::max(c->cap[1], p.kept_c);
+      ls.len[0] = p.kept_s;
+      ls.len[1] = p.kept_c;
+    }
+    c->limits.cand_stride = (cand_max + 3) & ~3;
+    c->limits.kept_stride = (kept_max + 3) & ~3;
+    c->limits.max_new = new_max;
+  }
+  c->layers.assign(cfg->n_layers, LayerState());
+  const int bh = cfg->batch * cfg->n_heads;
+  std::vector<int32_t> row_off((size_t)cfg->n_layers * bh);
+  size_t total_rows = 0;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    size_t rows = 0;
+    int n_ctx = 0;
+    for (int b = 0; b < cfg->batch; ++b)
+      for (int h = 0; h < cfg->n_heads; ++h) {
+        const int t = c->mask[(size_t)l * cfg->n_heads + h];
+        row_off[(size_t)l * bh + b * cfg->n_heads + h] = (int32_t)rows;
+        rows += c->cap[t];
+        if (b == 0) n_ctx += t;
+      }
+    if (rows > (1ull << 30)) { delete c; return fail(HACK_ERR_UNSUPPORTED, "layer plane too large"); }
+    c->n_ctx_heads.push_back(n_ctx);
+    c->layer_rows.push_back(rows);
+    c->layer_row_base.push_back(total_rows);
+    total_rows += rows;
+  }
+  c->row_off_host = row_off;
+  const size_t row_bytes = (size_t)cfg->head_dim * c->elt;
+  const size_t pad_rows = 256;    // slack after the last layer so that tiled reads stay inside
+  c->reserved_bytes = 2 * total_rows * row_bytes;
+
+  auto bail = [&](hack_status_t s) { hack_free_cache(c); return s; };
+#define HACK_TRY(call)                                                    \
+  do {                                                                    \
+    cudaError_t e_ = (call);                                              \
+    if (e_ != cudaSuccess) {                                              \
+      set_error(std::string(#call) + ": " + cudaGetErrorString(e_));      \
+      return bail(e_ == cudaErrorMemoryAllocation ? HACK_ERR_OOM : HACK_ERR_CUDA); \
+    }                                                                     \
+  } while (0)
+  HACK_TRY(cudaMalloc(&c->k_all, (total_rows + pad_rows) * row_bytes));
+  HACK_TRY(cudaMalloc(&c->v_all, (total_rows + pad_rows) * row_bytes));
+  HACK_TRY(cudaMalloc(&c->pos_all, (total_rows + pad_rows) * sizeof(int32_t)));
+  HACK_TRY(cudaMemset(c->k_all, 0, (total_rows + pad_rows) * row_bytes));
+  HACK_TRY(cudaMemset(c->v_all, 0, (total_rows + pad_rows) * row_bytes));
+  HACK_TRY(cudaMemset(c->pos_all, 0, (total_rows + pad_rows) * sizeof(int32_t)));
+  HACK_TRY(cudaMalloc(&c->row_off, row_off.size() * sizeof(int32_t)));
+  HACK_TRY(cudaMemcpy(c->row_off, row_off.data(), row_off.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+  HACK_TRY(cudaMalloc(&c->mask_dev, c->mask.size()));
+  HACK_TRY(cudaMemcpy(c->mask_dev, c->mask.data(), c->mask.size(), cudaMemcpyHostToDevice));
+  HACK_TRY(cudaMalloc(&c->scores, (size_t)bh * c->limits.cand_stride * sizeof(float)));
+  HACK_TRY(cudaMalloc(&c->idx, (size_t)bh * c->limits.kept_stride * sizeof(int32_t)));
+  c->scratch.max_chunks = (c->limits.cand_stride + hack::kScoreChunk - 1) / hack::kScoreChunk;
+  HACK_TRY(cudaMalloc(&c->scratch.logits, (size_t)bh * hack::kMaxObs * c->limits.cand_stride * sizeof(float)));
+  HACK_TRY(cudaMalloc(&c->scratch.partials, (size_t)bh * c->scratch.max_chunks * hack::kMaxObs * 2 * sizeof(float)));
+  HACK_TRY(cudaMalloc(&c->status, sizeof(int)));
+  HACK_TRY(cudaMemset(c->status, 0, sizeof(int)));
+  HACK_TRY(cudaDeviceSynchronize());
+#undef HACK_TRY
+  *out = c;
+  return HACK_OK;
+}
+
+hack_status_t hack_free_cache(hack_cache_t* c) {
+  if (!c) return HACK_OK;
+  cudaSetDevice(c->cfg.device);
+  cudaDeviceSynchronize();
+  cudaFree(c->k_all); cudaFree(c->v_all); cudaFree(c->pos_all); cudaFree(c->row_off);
+  cudaFree(c->mask_dev); cudaFree(c->scores); cudaFree(c->idx);
+  cudaFree(c->scratch.logits); cudaFree(c->scratch.partials); cudaFree(c->status);
+  for (int i = 0; i < 4; ++i) cudaFree(c->stage[i]);
+  delete c;
+  return HACK_OK;
+}
+
+hack_status_t hack_reset(hack_cache_t* c) {
+  if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
+  for (auto& ls : c->layers) ls = LayerState();
+  c->peak_bytes = 0;
+  return HACK_OK;
+}
+
+hack_status_t hack_get_limits(const hack_cache_t* c, hack_limits_t* out) {
+  if (!c || !out) return fail(HACK_ERR_INVALID_ARG, "cache or out is NULL");
+  *out = c->limits;
+  return HACK_OK;
+}
+
+hack_status_t hack_step_info(const hack_cache_t* c, int32_t layer, int32_t scale, hack_step_info_t* out) {
+  if (!out) return fail(HACK_ERR_INVALID_ARG, "out is NULL");
+  if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
+  if (layer < 0 || layer >= c->cfg.n_layers) return fail(HACK_ERR_INVALID_ARG, "layer out of range");
+  if (scale < 0 || scale >= c->cfg.n_scales) return fail(HACK_ERR_INVALID_ARG, "scale out of range");
+  const LayerState& ls = c->layers[layer];
+  if (scale != ls.next_scale || ls.phase != 0) return fail(HACK_ERR_STATE, "scale is not this layer's next step");
+  plan_step(c, ls, scale, out);
+  return HACK_OK;
+}
+
+hack_status_t hack_score(hack_cache_t* c, int32_t layer, int32_t scale, const void* q,
+                         const void* k_new, float* scores, void* stream) {
+  hack_status_t s = check_step(c, layer, scale, 0);
+  if (s != HACK_OK) return s;
+  if (!q || !k_new || !scores) return fail(HACK_ERR_INVALID_ARG, "q, k_new or scores is NULL");
+  if (misaligned(q) || misaligned(k_new) || misaligned(scores)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
+  hack_step_info_t p;
+  plan_step(c, c->layers[layer], scale, &p);
+  const hack::StepArgs a = make_args(c, layer, scale, p);
+  const int n = hack::launch_score(a, c->cfg.dtype, q, k_new, scores, c->scratch, (cudaStream_t)stream);
+  if (n < 0) return fail(HACK_ERR_CUDA, "score launch failed");
+  c->launches += n;
+  return HACK_OK;
+}
+
+hack_status_t hack_select(hack_cache_t* c, int32_t layer, int32_t scale, const float* scores,
+                          int32_t* idx, int32_t* kept_out, void* stream) {
+  hack_status_t s = check_step(c, layer, scale, 0);
+  if (s != HACK_OK) return s;
+  if (!scores || !idx) return fail(HACK_ERR_INVALID_ARG, "scores or idx is NULL");
+  hack_step_info_t p;
+  plan_step(c, c->layers[layer], scale, &p);
+  const hack::StepArgs a = make_args(c, layer, scale, p);
+  const int n = hack::launch_select(a, scores, idx, kept_out, (cudaStream_t)stream);
+  if (n < 0) return fail(HACK_ERR_CUDA, "select launch failed");
+  c->launches += n;
+  return HACK_OK;
+}
+
+hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const int32_t* idx,
+                           const void* k_new, const void* v_new, void* stream) {
+  hack_status_t s = check_step(c, layer, scale, 0);
+  if (s != HACK_OK) return s;
+  if (!idx || !k_new || !v_new) return fail(HACK_ERR_INVALID_ARG, "idx, k_new or v_new is NULL");
+  if (misaligned(k_new) || misaligned(v_new)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
+  hack_step_info_t p;
+  plan_step(c, c->layers[layer], scale, &p);
+  const hack::StepArgs a = make_args(c, layer, scale, p);
+  const int n = hack::launch_compact(a, c->cfg.dtype, idx, 1, k_new, v_new, (cudaStream_t)stream);
+  if (n < 0) return fail(HACK_ERR_CUDA, "compact launch failed");
+  c->launches += n;
+  advance_after_compact(c, layer, p);
+  return HACK_OK;
+}
+
+static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void* q, void* out, cudaStream_t st) {
+  // lengths are already those after compaction
+  LayerState& ls = c->layers[layer];
+  hack_step_info_t p{};
+  p.n_new = c->n_tok[scale];
+  p.kept_s = ls.len[0];
+  p.kept_c = ls.len[1];
+  p.n_obs_rows = std::min(c->cfg.n_obs, p.n_new);
+  const hack::StepArgs a = make_args(c, layer, scale, p);
+  const int n = hack::launch_attend(a, c->cfg.dtype, q, out, st);
+  if (n < 0) return fail(HACK_ERR_CUDA, "attend launch failed");
+  c->launches += n;
+  ls.phase = 0;
+  ls.next_scale = scale + 1;
+  return HACK_OK;
+}
+
+hack_status_t hack_attend(hack_cache_t* c, int32_t layer, int32_t scale, const void* q, void* out, void* stream) {
+  hack_status_t s = check_step(c, layer, scale, 1);
+  if (s != HACK_OK) return s;
+  if (!q || !out) return fail(HACK_ERR_INVALID_ARG, "q or out is NULL");
+  if (misaligned(q) || misaligned(out)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
+  return attend_impl(c, layer, scale, q, out, (cudaStream_t)stream);
+}
+
+hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, const void* q,
+                              const void* k, const void* v, void* out, void* stream) {
+  hack_status_t s = check_step(c, layer, scale, 0);
+  if (s != HACK_OK) return s;
+  if (!q || !k || !v || !out) return fail(HACK_ERR_INVALID_ARG, "q, k, v or out is NULL");
+  if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(out)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
+  cudaStream_t st = (cudaStream_t)stream;
+  hack_step_info_t p;
+  plan_step(c, c->layers[layer], scale, &p);
+  const hack::StepArgs a = make_args(c, layer, scale, p);
+  const bool any = p.triggered_c || p.triggered_s;
+  int n = 0, r;
+  if (any) {
+    if ((r = hack::launch_score(a, c->cfg.dtype, q, k, c->scores, c->scratch, st)) < 0) return fail(HACK_ERR_CUDA, "score launch failed");
+    n += r;
+    if ((r = hack::launch_select(a, c->scores, c->idx, nullptr, st)) < 0) return fail(HACK_ERR_CUDA, "select launch failed");
+    n += r;
+  }
+  if ((r = hack::launch_compact(a, c->cfg.dtype, any ? c->idx : nullptr, any ? 1 : 0, k, v, st)) < 0) return fail(HACK_ERR_CUDA, "compact launch failed");
+  n += r;
+  c->launches += n;
+  advance_after_compact(c, layer, p);
+  return attend_impl(c, layer, scale, q, out, st);
+}
+
+hack_status_t hack_scale_step_host(hack_cache_t* c, int32_t layer, int32_t scale, const void* q_host,
+                                   const void* k_host, const void* v_host, void* out_host, void* stream) {
+  hack_status_t s = check_step(c, layer, scale, 0);
+  if (s != HACK_OK) return s;
+  if (!q_host || !k_host || !v_host || !out_host) return fail(HACK_ERR_INVALID_ARG, "a host buffer is NULL");
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t full = (size_t)c->cfg.batch * c->cfg.n_heads * c->limits.max_new * c->cfg.head_dim * c->elt;
+  if (!c->stage[0]) {
+    for (int i = 0; i < 4; ++i) {
+      cudaError_t e = cudaMalloc(&c->stage[i], full);
+      if (e != cudaSuccess) {
+        for (int j = 0; j < 4; ++j) { cudaFree(c->stage[j]); c->stage[j] = nullptr; }
+        set_error(std::string("staging cudaMalloc: ") + cudaGetErrorString(e));
+        return HACK_ERR_OOM;
+      }
+    }
+  }
+  const size_t bytes = (size_t)c->cfg.batch * c->cfg.n_heads * c->n_tok[scale] * c->cfg.head_dim * c->elt;
+  HACK_CUDA(cudaMemcpyAsync(c->stage[0], q_host, bytes, cudaMemcpyHostToDevice, st));
+  HACK_CUDA(cudaMemcpyAsync(c->stage[1], k_host, bytes, cudaMemcpyHostToDevice, st));
+  HACK_CUDA(cudaMemcpyAsync(c->stage[2], v_host, bytes, cudaMemcpyHostToDevice, st));
+  s = hack_scale_step(c, layer, scale, c->stage[0], c->stage[1], c->stage[2], c->stage[3], stream);
+  if (s != HACK_OK) return s;
+  HACK_CUDA(cudaMemcpyAsync(out_host, c->stage[3], bytes, cudaMemcpyDeviceToHost, st));
+  return HACK_OK;
+}
+
+hack_status_t hack_get_lengths(const hack_cache_t* c, int32_t layer, int32_t* host_out) {
+  if (!c || !host_out) return fail(HACK_ERR_INVALID_ARG, "cache or host_out is NULL");
+  if (layer < 0 || layer >= c->cfg.n_layers) return fail(HACK_ERR_INVALID_ARG, "layer out of range");
+  const LayerState& ls = c->layers[layer];
+  for (int b = 0; b < c->cfg.batch; ++b)
+    for (int h = 0; h < c->cfg.n_heads; ++h)
+      host_out[b * c->cfg.n_heads + h] = ls.len[c->mask[(size_t)layer * c->cfg.n_heads + h]];
+  return HACK_OK;
+}
+
+hack_status_t hack_read_head(hack_cache_t* c, int32_t layer, int32_t b, int32_t h, int32_t which,
+                             void* host_out, size_t bytes) {
+  if (!c || !host_out) return fail(HACK_ERR_INVALID_ARG, "cache or host_out is NULL");
+  if (layer < 0 || layer >= c->cfg.n_layers || b < 0 || b >= c->cfg.batch || h < 0 || h >= c->cfg.n_heads)
+    return fail(HACK_ERR_INVALID_ARG, "layer, b or h out of range");
+  if (which < 0 || which > 2) return fail(HACK_ERR_INVALID_ARG, "which must be 0, 1 or 2");
+  const int t = c->mask[(size_t)layer * c->cfg.n_heads + h];
+  const size_t len = c->layers[layer].len[t];
+  const size_t row_bytes = (size_t)c->cfg.head_dim * c->elt;
+  const size_t need = which == 2 ? len * sizeof(int32_t) : len * row_bytes;
+  if (bytes < need) return fail(HACK_ERR_INVALID_ARG, "host_out is too small for the stored length");
+  const size_t off = c->row_off_host[((size_t)layer * c->cfg.batch + b) * c->cfg.n_heads + h];
+  HACK_CUDA(cudaDeviceSynchronize());
+  const size_t row = c->layer_row_base[layer] + off;
+  if (need == 0) return HACK_OK;
+  if (which == 2) HACK_CUDA(cudaMemcpy(host_out, c->pos_all + row, need, cudaMemcpyDeviceToHost));
+  else HACK_CUDA(cudaMemcpy(host_out, (which == 0 ? c->k_all : c->v_all) + row * row_bytes, need, cudaMemcpyDeviceToHost));
+  return HACK_OK;
+}
+
+hack_status_t hack_kv_bytes(const hack_cache_t* c, size_t* live, size_t* peak, size_t* reserved) {
+  if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
+  if (live) *live = live_bytes(c);
+  if (peak) *peak = c->peak_bytes;
+  if (reserved) *reserved = c->reserved_bytes;
+  return HACK_OK;
+}
+
+hack_status_t hack_launch_count(const hack_cache_t* c, uint64_t* launches) {
+  if (!c || !launches) return fail(HACK_ERR_INVALID_ARG, "cache or launches is NULL");
+  *launches = c->launches;
+  return HACK_OK;
+}
+
+hack_status_t hack_poll_status(hack_cache_t* c, void* stream) {
+  if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
+  HACK_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  int word = 0;
+  HACK_CUDA(cudaMemcpy(&word, c->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (word != 0) {
+    HACK_CUDA(cudaMemset(c->status, 0, sizeof(int)));
+    set_error("a bounded device-side wait expired (status word " + std::to_string(word) + ")");
+    return HACK_ERR_TIMEOUT;
+  }
+  return HACK_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,60 @@
+// Internal declarations shared by the host API and the kernel translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "hack.h"
+
+namespace hack {
+
+constexpr int kMaxObs = 32;        // rows of the observation window the kernels are built for
+constexpr int kScoreChunk = 128;   // candidate keys per CTA in the SIMT scoring pass
+
+// Everything a kernel needs to know about one (layer, scale) step.  Passed by value.
+// Per-type arrays are indexed by the head's mask byte: [0] structural, [1] contextual.
+struct StepArgs {
+  int n_heads, batch, head_dim;
+  int n_new;            // N_k
+  int stored[2];        // L before the step
+  int cand[2];          // T' = L + N_k
+  int kept[2];          // length after the step
+  int trig[2];          // compression triggered for this type
+  int n_obs_rows;       // min(N_obs, N_k)
+  float sm_scale;
+  int t_init;           // tokens in the always-kept leading scales (structural heads)
+  int protect_new;      // structural heads: the new scale's tokens are protected
+  int pos_base;         // global position of the new scale's first token (T_{k-1})
+  int cand_stride, kept_stride;
+  const uint8_t* is_ctx;   // device, [n_heads] of this layer
+  const int32_t* row_off;  // device, [batch*n_heads] first row of each head in the planes
+  void* k_plane;           // device, [rows, head_dim] of this layer
+  void* v_plane;
+  int32_t* pos_plane;      // device, [rows]
+  int* status;             // device status word
+};
+
+struct Scratch {
+  float* logits;    // [batch*n_heads, kMaxObs, cand_stride]
+  float* partials;  // [batch*n_heads, max_chunks, kMaxObs, 2]  (row max, row sum per chunk)
+  int max_chunks;
+};
+
+// Kernel launchers (each returns the number of kernels it enqueued, or -1 on a launch error).
+int launch_score(const StepArgs& a, int dtype, const void* q, const void* k_new, float* scores,
+                 const Scratch& s, cudaStream_t st);
+int launch_select(const StepArgs& a, const float* scores, int32_t* idx, int32_t* kept_out,
+                  cudaStream_t st);
+// idx == nullptr: every head appends (keeps all candidates).  idx_all != 0: idx rows are valid for
+// heads that are not triggered as well (identity lists written by launch_select).
+int launch_compact(const StepArgs& a, int dtype, const int32_t* idx, int idx_all, const void* k_new,
+                   const void* v_new, cudaStream_t st);
+int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st);
+
+void set_error(const std::string& msg);
+
+}  // namespace hack

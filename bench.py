@@ -1,0 +1,451 @@
+#!/usr/bin/env python
+"""Benchmark of the per-scale decoding hot path (score -> select -> compact -> attend).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config I]
+
+A "step" is one pass of the whole hot path over one batch of synthetic input: the full decoding
+loop of one image batch, every layer at every scale, each (layer, scale) served by one
+hack_scale_step call.  The default workload is config 3 (Infinity-2B-shaped stack, 1024x1024,
+13 scales, batch 2, bf16, budget 30 %), the configuration the roofline target is quoted on.
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from workloads import SyntheticQKV, get_config  # noqa: E402
+
+METRIC = "scale-step tokens/s (score+select+compact+attend)"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------- work model
+def step_work(info, cfg, n_ctx_heads, persist=True):
+    """Algorithmic FLOPs and bytes of one (layer, scale) step from its length plan."""
+    D, e, b, H = cfg.head_dim, (4 if cfg.dtype == "f32" else 2), cfg.batch, cfg.n_heads
+    n_c, n_s = b * n_ctx_heads, b * (H - n_ctx_heads)
+    kept = n_c * info.kept_c + n_s * info.kept_s
+    cand = n_c * info.cand_c * info.triggered_c + n_s * info.cand_s * info.triggered_s
+    attend_flops = 4.0 * info.n_new * D * kept
+    score_flops = 2.0 * info.n_obs_rows * D * cand
+    nbytes = cand * (D * e + 8) + 2 * kept * 2 * D * e + 2 * info.n_new * H * b * D * e
+    return attend_flops, score_flops, float(nbytes)
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.index)],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    parts = [p.strip() for p in line.split(",")]
+                    if len(parts) < 7:
+                        continue
+                    try:
+                        sm.append(float(parts[0]))
+                        smax.append(float(parts[1]))
+                    except ValueError:
+                        continue
+                    for n, v in zip(names, parts[3:7]):
+                        if v.lower().startswith("active"):
+                            reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ----------------------------------------------------------------------------- oracle arm
+_ORACLE_INPUTS = {}
+
+
+def oracle_sample_run(cfg, n_pairs: int):
+    """Time the CPU oracle, as it stands, on layer 0 of the workload: all scales, n_pairs of the
+    (batch, head) pairs.  Returns (seconds, fraction of one full step covered, threads)."""
+    import numpy as np
+    from oracle import hack_oracle as ho
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    one = cfg.with_layers(1)
+    gen = SyntheticQKV(one)
+    mask = gen.head_is_contextual.numpy()
+    pairs_all = [(b, h) for b in range(cfg.batch) for h in range(cfg.n_heads)]
+    # alternate contextual / structural heads so the sample has the workload's mix
+    ctx = [p for p in pairs_all if mask[0, p[1]]]
+    stc = [p for p in pairs_all if not mask[0, p[1]]]
+    n_c = max(1, round(n_pairs * len(ctx) / len(pairs_all))) if ctx else 0
+    pairs = ctx[:n_c] + stc[: n_pairs - n_c]
+    if cfg.index not in _ORACLE_INPUTS:          # generated once, outside the timed part
+        _ORACLE_INPUTS[cfg.index] = [tuple(t.to(torch.float64).numpy() for t in gen.qkv(0, k))
+                                     for k in range(cfg.n_scales)]
+    inputs = _ORACLE_INPUTS[cfg.index]
+    orc = ho.HackOracle(1, cfg.n_heads, cfg.batch, cfg.head_dim, cfg.sides, mask, cfg.budget_c,
+                        cfg.budget_s, n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales)
+    t0 = time.perf_counter()
+    for k in range(cfg.n_scales):
+        q, kk, v = inputs[k]
+        orc.scale_step(0, k, q, kk, v, heads=pairs)
+    dt = time.perf_counter() - t0
+    frac = (len(pairs) / len(pairs_all)) / cfg.n_layers
+    return dt, frac, threads, len(pairs)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = get_config(args.config)
+    tokens = cfg.batch * cfg.total_tokens
+    n_pairs = args.oracle_pairs
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_run(cfg, 2)
+    times = []
+    for _ in range(args.steps):
+        dt, frac, threads, used = oracle_sample_run(cfg, n_pairs)
+        times.append(dt / frac)
+    sec = sum(times) / len(times)
+    value = tokens / sec
+    sample = (f"layer 0 of {cfg.n_layers}, all {cfg.n_scales} scales, {used} of "
+              f"{cfg.batch * cfg.n_heads} (batch, head) pairs; time scaled by 1/{frac:.6f}")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": f"config {cfg.index}: {cfg.name}", "tokens_per_step": tokens,
+                   "budget": cfg.budget_total, "budget_c": cfg.budget_c, "budget_s": cfg.budget_s},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import paper_2504_09261_b200 as hb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+
+    cfg = get_config(args.config)
+    if args.layers:
+        cfg = cfg.with_layers(args.layers)
+    L, K = cfg.n_layers, cfg.n_scales
+    gen = SyntheticQKV(cfg, device=dev, seed_offset=rank)      # each rank decodes its own images
+    mask = gen.head_is_contextual
+    n_ctx = [int(mask[l].sum()) for l in range(L)]
+    dtype_id = hb.HACK_F32 if cfg.dtype == "f32" else hb.HACK_BF16
+
+    def new_cache(bc, bs):
+        return hb.HackCache(L, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides, dtype_id, mask.numpy(),
+                            bc, bs, n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, device=local)
+
+    cache = new_cache(cfg.budget_c, cfg.budget_s)
+    # inputs resident in HBM: every (layer, scale) has its own Q, K, V (ranks draw different images)
+    qkv = [[None] * K for _ in range(L)]
+    in_bytes = 0
+    for l in range(L):
+        for k in range(K):
+            qkv[l][k] = gen.qkv(l, k)
+            in_bytes += sum(t.numel() * t.element_size() for t in qkv[l][k])
+    outs = [torch.empty_like(qkv[0][k][0]) for k in range(K)]
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+
+    def loop(c, scale_events=None):
+        c.hack_reset()
+        for k in range(K):
+            for l in range(L):
+                q, kk, v = qkv[l][k]
+                c.hack_scale_step(l, k, q, kk, v, outs[k], sh)
+            if scale_events is not None:
+                scale_events[k].record(stream)
+
+    def timed(c, steps, warmup, per_scale=False):
+        for _ in range(warmup):
+            loop(c)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ev0 = torch.cuda.Event(enable_timing=True)
+        ev1 = torch.cuda.Event(enable_timing=True)
+        sev = [[torch.cuda.Event(enable_timing=True) for _ in range(K)] for _ in range(steps)] if per_scale else None
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)] if per_scale else None
+        ev0.record(stream)
+        for s in range(steps):
+            if per_scale:
+                starts[s].record(stream)
+            loop(c, sev[s] if per_scale else None)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1)
+        scale_ms = None
+        if per_scale:
+            scale_ms = [0.0] * K
+            for s in range(steps):
+                prev = starts[s]
+                for k in range(K):
+                    scale_ms[k] += prev.elapsed_time(sev[s][k]) / steps
+                    prev = sev[s][k]
+        return ms, scale_ms
+
+    launches0 = cache.hack_launch_count()
+    sampler = ClockSampler(local)
+    sampler.start()
+    total_ms, scale_ms = timed(cache, args.steps, args.warmup, per_scale=True)
+    clocks = sampler.stop()
+    launches_per_step = (cache.hack_launch_count() - launches0) // (args.steps + args.warmup)
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    tokens = cfg.batch * cfg.total_tokens
+    value = world * tokens / (ms_per_step * 1e-3)
+    live, peak, reserved = cache.hack_kv_bytes()
+
+    # ---- work model and roofline of the loop
+    peaks, peak_kind = load_peaks()
+    hbm = peaks["hbm_gbs"] * 1e9
+    tf_sus = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12
+    infos = []
+    walker = hb.HackCache(1, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides, dtype_id, mask[0].numpy(),
+                          cfg.budget_c, cfg.budget_s, n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales,
+                          device=local)
+    # lengths depend on the head type only, so layer 0's plan holds for every layer
+    dq = torch.zeros((cfg.batch, cfg.n_heads, max(cfg.tokens_per_scale), cfg.head_dim),
+                     dtype=qkv[0][0][0].dtype, device=dev)
+    for k in range(K):
+        infos.append(walker.hack_step_info(0, k))
+        walker.hack_scale_step(0, k, dq, dq, dq, dq, sh)
+    torch.cuda.synchronize()
+    walker.close()
+    attend_fl = score_fl = byt = 0.0
+    t_roof = 0.0
+    per_scale = []
+    for k in range(K):
+        a_k = s_k = b_k = roof_k = 0.0
+        for l in range(L):
+            a, s, by = step_work(infos[k], cfg, n_ctx[l])
+            a_k += a
+            s_k += s
+            b_k += by
+            roof_k += max((a + s) / tf_sus, by / hbm)
+        attend_fl += a_k
+        score_fl += s_k
+        byt += b_k
+        t_roof += roof_k
+        per_scale.append({
+            "scale": k, "n_new": infos[k].n_new, "kept_c": infos[k].kept_c, "kept_s": infos[k].kept_s,
+            "ms": round(scale_ms[k], 4),
+            "tokens_per_s": round(cfg.batch * infos[k].n_new / (scale_ms[k] * 1e-3), 1),
+            "roofline_ms": round(roof_k * 1e3, 4),
+            "roofline_frac": round(roof_k * 1e3 / scale_ms[k], 4),
+        })
+
+    # ---- per-stage device time (second pass, stage events on) -> roofline of the dominant kernel
+    stage = None
+    roofline = None
+    if rank == 0:
+        cache.hack_stage_timing(True)
+        n_prof = 2
+        for _ in range(n_prof):
+            loop(cache)
+        st = cache.hack_stage_times()
+        cache.hack_stage_timing(False)
+        stage = {k: {"ms_per_step": v[0] / n_prof, "launches_per_step": v[1] // n_prof} for k, v in st.items()}
+        att_ms = stage["attend"]["ms_per_step"]
+        att_n = max(stage["attend"]["launches_per_step"], 1)
+        achieved = attend_fl / (att_ms * 1e-3) / 1e12
+        peak_tf = tf_sus / 1e12
+        if cfg.dtype == "f32":
+            peak_tf = None
+        roofline = {
+            "kernel": "attend", "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
+            "frac": (achieved / peak_tf) if peak_tf else None, "traffic": None,
+            "peak_source": f"bf16_tflops_sustained of {peak_kind}",
+            "flops_per_launch": attend_fl / att_n, "avg_launch_ms": att_ms / att_n,
+            "launches_per_step": att_n,
+        }
+
+    # ---- e2e: same loop through the host-buffer entry point (pinned host memory)
+    e2e = None
+    if not args.no_e2e:
+        host = [[tuple(t.cpu().pin_memory() for t in qkv[l][k]) for k in range(K)] for l in range(L)]
+        host_out = [torch.empty_like(host[0][k][0]).pin_memory() for k in range(K)]
+        c2 = new_cache(cfg.budget_c, cfg.budget_s)
+
+        def loop_host():
+            c2.hack_reset()
+            for k in range(K):
+                for l in range(L):
+                    q, kk, v = host[l][k]
+                    c2.hack_scale_step_host(l, k, q, kk, v, host_out[k], sh)
+
+        for _ in range(2):
+            loop_host()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_e2e = max(1, min(args.steps, 3))
+        e0.record(stream)
+        for _ in range(n_e2e):
+            loop_host()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / n_e2e
+        if dist is not None:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        e2e = {"value": world * tokens / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+               "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": in_bytes // 3}
+        c2.close()
+        del host, host_out
+
+    # ---- uncompressed comparison run (same call, budgets = T_K)
+    full = None
+    if rank == 0 and not args.no_full:
+        cf = new_cache(cfg.total_tokens, cfg.total_tokens)
+        ms_f, _ = timed(cf, 1, 1)
+        _, peak_f, res_f = cf.hack_kv_bytes()
+        full = {"ms_per_step": ms_f, "tokens_per_s": tokens / (ms_f * 1e-3), "kv_bytes_peak": peak_f,
+                "speedup_of_budgeted_run": ms_f / ms_per_step}
+        cf.close()
+
+    # ---- CPU oracle on the host cores (rank 0, N = 1)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        base_cfg = get_config(args.config)
+        dt, frac, threads, used = oracle_sample_run(base_cfg, args.oracle_pairs)
+        cpu = {"value": base_cfg.batch * base_cfg.total_tokens / (dt / frac), "unit": UNIT, "cores": threads,
+               "kind": "oracle", "seconds_measured": dt,
+               "sample": (f"layer 0 of {base_cfg.n_layers}, all {base_cfg.n_scales} scales, {used} of "
+                          f"{base_cfg.batch * base_cfg.n_heads} (batch, head) pairs; time scaled by 1/{frac:.6f}")}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "config": {
+                "workload": f"config {cfg.index}: {cfg.name}", "n_layers": L, "n_heads": cfg.n_heads,
+                "head_dim": cfg.head_dim, "batch": cfg.batch, "scales": list(cfg.sides),
+                "tokens_per_step": tokens, "budget": cfg.budget_total, "budget_c": cfg.budget_c,
+                "budget_s": cfg.budget_s, "calls_per_step": L * K,
+                "l2": f"inputs larger than L2 ({in_bytes / 1e9:.2f} GB of Q/K/V walked once per step)",
+                "sharding": "independent image batches per GPU, no collective in the path",
+            },
+            "roofline": roofline,
+            "loop_roofline": {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_per_step,
+                              "flops": attend_fl + score_fl, "bytes": byt, "peaks": peak_kind},
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks, "stages": stage, "per_scale": per_scale,
+            "kv_bytes": {"live": live, "peak": peak, "reserved": reserved,
+                         "full_cache": 2 * cfg.total_tokens * cfg.head_dim * (4 if cfg.dtype == "f32" else 2)
+                         * cfg.n_heads * L * cfg.batch},
+            "full_cache_run": full,
+        }
+        print(json.dumps(line))
+    cache.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=3)
+    ap.add_argument("--layers", type=int, default=0, help="restrict the stack (debugging only)")
+    ap.add_argument("--oracle-pairs", type=int, default=8)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-full", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -171,6 +171,13 @@ HACK_API hack_status_t hack_read_head(hack_cache_t* cache, int32_t layer, int32_
 HACK_API hack_status_t hack_kv_bytes(const hack_cache_t* cache, size_t* live, size_t* peak, size_t* reserved);
 /* Number of the library's own kernel launches enqueued through this cache since init. */
 HACK_API hack_status_t hack_launch_count(const hack_cache_t* cache, uint64_t* launches);
+/* Per-stage device timing for benchmarks.  enable != 0: from now on every stage's launches are
+ * bracketed by two CUDA events on the caller's stream (a few microseconds of overhead per
+ * stage); accumulators are cleared.  Synchronises the device. */
+HACK_API hack_status_t hack_stage_timing(hack_cache_t* cache, int32_t enable);
+/* Synchronises the device and returns the accumulated device time in ms and the number of kernel
+ * launches per stage since timing was enabled: [0] score, [1] select, [2] compact, [3] attend. */
+HACK_API hack_status_t hack_stage_times(hack_cache_t* cache, double* ms, uint64_t* launches);
 /* Synchronises `stream`, then reports the device status word: HACK_OK, or HACK_ERR_TIMEOUT if a
  * bounded device-side wait gave up (the word is cleared by the call). */
 HACK_API hack_status_t hack_poll_status(hack_cache_t* cache, void* stream);

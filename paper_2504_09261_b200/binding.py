@@ -22,7 +22,7 @@ EXPORTS = (
     "hack_split_budget", "hack_init_cache", "hack_free_cache", "hack_reset", "hack_get_limits",
     "hack_step_info", "hack_score", "hack_select", "hack_compact", "hack_attend", "hack_scale_step",
     "hack_scale_step_host", "hack_get_lengths", "hack_read_head", "hack_kv_bytes",
-    "hack_launch_count", "hack_poll_status", "hack_last_error",
+    "hack_launch_count", "hack_stage_timing", "hack_stage_times", "hack_poll_status", "hack_last_error",
 )
 
 
@@ -55,7 +55,7 @@ class HackError(RuntimeError):
 def _load() -> C.CDLL:
     if not os.path.exists(_LIB_PATH):
         raise ImportError(
-            f"{_LIB_PATH} is missing: build it with `python -m paper_2504_09261_b200.build` "
+            f"{_LIB_PATH} is missing: build it with `python paper_2504_09261_b200/build.py` "
             "(there is no fallback implementation)")
     lib = C.CDLL(_LIB_PATH)
     vp, i32 = C.c_void_p, C.c_int32
@@ -79,6 +79,8 @@ def _load() -> C.CDLL:
         "hack_kv_bytes": [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)],
         "hack_launch_count": [vp, C.POINTER(C.c_uint64)],
         "hack_poll_status": [vp, vp],
+        "hack_stage_timing": [vp, i32],
+        "hack_stage_times": [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)],
     }
     for name, args in sigs.items():
         fn = getattr(lib, name)
@@ -198,6 +200,16 @@ class HackCache:
         n = C.c_uint64()
         _check(lib.hack_launch_count(self._h, C.byref(n)))
         return n.value
+
+    def hack_stage_timing(self, enable: bool) -> None:
+        _check(lib.hack_stage_timing(self._h, 1 if enable else 0))
+
+    def hack_stage_times(self):
+        ms = (C.c_double * 4)()
+        n = (C.c_uint64 * 4)()
+        _check(lib.hack_stage_times(self._h, ms, n))
+        names = ("score", "select", "compact", "attend")
+        return {k: (ms[i], n[i]) for i, k in enumerate(names)}
 
     def hack_poll_status(self, stream=None) -> None:
         _check(lib.hack_poll_status(self._h, _ptr(stream)))

@@ -1,6 +1,6 @@
 """Build the C-ABI shared library (sm_100a) with nvcc, in-tree.
 
-    python -m paper_2504_09261_b200.build [--force] [--verbose]
+    python paper_2504_09261_b200/build.py [--force] [--verbose]
 
 Produces paper_2504_09261_b200/lib/libhack_b200.so from csrc/*.cu.  Object files are cached under
 paper_2504_09261_b200/_build and rebuilt when a source or header is newer.

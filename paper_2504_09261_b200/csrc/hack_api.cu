@@ -57,6 +57,14 @@ struct hack_cache {
   unsigned char* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging
   size_t reserved_bytes = 0, peak_bytes = 0;
   uint64_t launches = 0;
+  // optional per-stage device timing (score, select, compact, attend)
+  bool timing = false;
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_used = 0;
+  struct Span { int stage; size_t e0, e1; int launches; };
+  std::vector<Span> spans;
+  double stage_ms[4] = {0, 0, 0, 0};
+  uint64_t stage_launches[4] = {0, 0, 0, 0};
 };
 
 namespace {
@@ -153,6 +161,30 @@ hack_status_t check_step(const hack_cache* c, int layer, int scale, int want_pha
                                            : "this scale is already compacted; call hack_attend");
   return HACK_OK;
 }
+
+// Brackets one stage's launches with two events when stage timing is on.
+struct StageScope {
+  hack_cache* c; cudaStream_t st; int stage; size_t e0 = 0; bool on;
+  StageScope(hack_cache* c_, cudaStream_t st_, int stage_) : c(c_), st(st_), stage(stage_), on(c_->timing) {
+    if (!on) return;
+    e0 = grab();
+    cudaEventRecord(c->ev_pool[e0], st);
+  }
+  size_t grab() {
+    if (c->ev_used == c->ev_pool.size()) {
+      cudaEvent_t e;
+      cudaEventCreate(&e);
+      c->ev_pool.push_back(e);
+    }
+    return c->ev_used++;
+  }
+  void done(int launches) {
+    if (!on) return;
+    const size_t e1 = grab();
+    cudaEventRecord(c->ev_pool[e1], st);
+    c->spans.push_back({stage, e0, e1, launches});
+  }
+};
 
 bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -316,6 +348,7 @@ hack_status_t hack_free_cache(hack_cache_t* c) {
   cudaFree(c->mask_dev); cudaFree(c->scores); cudaFree(c->idx);
   cudaFree(c->scratch.logits); cudaFree(c->scratch.partials); cudaFree(c->status);
   for (int i = 0; i < 4; ++i) cudaFree(c->stage[i]);
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   delete c;
   return HACK_OK;
 }
@@ -353,8 +386,10 @@ hack_status_t hack_score(hack_cache_t* c, int32_t layer, int32_t scale, const vo
   hack_step_info_t p;
   plan_step(c, c->layers[layer], scale, &p);
   const hack::StepArgs a = make_args(c, layer, scale, p);
+  StageScope ts(c, (cudaStream_t)stream, 0);
   const int n = hack::launch_score(a, c->cfg.dtype, q, k_new, scores, c->scratch, (cudaStream_t)stream);
   if (n < 0) return fail(HACK_ERR_CUDA, "score launch failed");
+  ts.done(n);
   c->launches += n;
   return HACK_OK;
 }
@@ -367,8 +402,10 @@ hack_status_t hack_select(hack_cache_t* c, int32_t layer, int32_t scale, const f
   hack_step_info_t p;
   plan_step(c, c->layers[layer], scale, &p);
   const hack::StepArgs a = make_args(c, layer, scale, p);
+  StageScope ts(c, (cudaStream_t)stream, 1);
   const int n = hack::launch_select(a, scores, idx, kept_out, (cudaStream_t)stream);
   if (n < 0) return fail(HACK_ERR_CUDA, "select launch failed");
+  ts.done(n);
   c->launches += n;
   return HACK_OK;
 }
@@ -382,8 +419,10 @@ hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const 
   hack_step_info_t p;
   plan_step(c, c->layers[layer], scale, &p);
   const hack::StepArgs a = make_args(c, layer, scale, p);
+  StageScope ts(c, (cudaStream_t)stream, 2);
   const int n = hack::launch_compact(a, c->cfg.dtype, idx, 1, k_new, v_new, (cudaStream_t)stream);
   if (n < 0) return fail(HACK_ERR_CUDA, "compact launch failed");
+  ts.done(n);
   c->launches += n;
   advance_after_compact(c, layer, p);
   return HACK_OK;
@@ -398,8 +437,10 @@ static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void
   p.kept_c = ls.len[1];
   p.n_obs_rows = std::min(c->cfg.n_obs, p.n_new);
   const hack::StepArgs a = make_args(c, layer, scale, p);
+  StageScope ts(c, st, 3);
   const int n = hack::launch_attend(a, c->cfg.dtype, q, out, st);
   if (n < 0) return fail(HACK_ERR_CUDA, "attend launch failed");
+  ts.done(n);
   c->launches += n;
   ls.phase = 0;
   ls.next_scale = scale + 1;
@@ -427,13 +468,25 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
   const bool any = p.triggered_c || p.triggered_s;
   int n = 0, r;
   if (any) {
-    if ((r = hack::launch_score(a, c->cfg.dtype, q, k, c->scores, c->scratch, st)) < 0) return fail(HACK_ERR_CUDA, "score launch failed");
-    n += r;
-    if ((r = hack::launch_select(a, c->scores, c->idx, nullptr, st)) < 0) return fail(HACK_ERR_CUDA, "select launch failed");
+    {
+      StageScope ts(c, st, 0);
+      if ((r = hack::launch_score(a, c->cfg.dtype, q, k, c->scores, c->scratch, st)) < 0) return fail(HACK_ERR_CUDA, "score launch failed");
+      ts.done(r);
+      n += r;
+    }
+    {
+      StageScope ts(c, st, 1);
+      if ((r = hack::launch_select(a, c->scores, c->idx, nullptr, st)) < 0) return fail(HACK_ERR_CUDA, "select launch failed");
+      ts.done(r);
+      n += r;
+    }
+  }
+  {
+    StageScope ts(c, st, 2);
+    if ((r = hack::launch_compact(a, c->cfg.dtype, any ? c->idx : nullptr, any ? 1 : 0, k, v, st)) < 0) return fail(HACK_ERR_CUDA, "compact launch failed");
+    ts.done(r);
     n += r;
   }
-  if ((r = hack::launch_compact(a, c->cfg.dtype, any ? c->idx : nullptr, any ? 1 : 0, k, v, st)) < 0) return fail(HACK_ERR_CUDA, "compact launch failed");
-  n += r;
   c->launches += n;
   advance_after_compact(c, layer, p);
   return attend_impl(c, layer, scale, q, out, st);
@@ -507,6 +560,31 @@ hack_status_t hack_kv_bytes(const hack_cache_t* c, size_t* live, size_t* peak, s
 hack_status_t hack_launch_count(const hack_cache_t* c, uint64_t* launches) {
   if (!c || !launches) return fail(HACK_ERR_INVALID_ARG, "cache or launches is NULL");
   *launches = c->launches;
+  return HACK_OK;
+}
+
+hack_status_t hack_stage_timing(hack_cache_t* c, int32_t enable) {
+  if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
+  HACK_CUDA(cudaDeviceSynchronize());
+  c->timing = enable != 0;
+  c->spans.clear();
+  c->ev_used = 0;
+  for (int i = 0; i < 4; ++i) { c->stage_ms[i] = 0; c->stage_launches[i] = 0; }
+  return HACK_OK;
+}
+
+hack_status_t hack_stage_times(hack_cache_t* c, double* ms, uint64_t* launches) {
+  if (!c || !ms || !launches) return fail(HACK_ERR_INVALID_ARG, "cache, ms or launches is NULL");
+  HACK_CUDA(cudaDeviceSynchronize());
+  for (const auto& sp : c->spans) {
+    float t = 0.f;
+    HACK_CUDA(cudaEventElapsedTime(&t, c->ev_pool[sp.e0], c->ev_pool[sp.e1]));
+    c->stage_ms[sp.stage] += t;
+    c->stage_launches[sp.stage] += sp.launches;
+  }
+  c->spans.clear();
+  c->ev_used = 0;
+  for (int i = 0; i < 4; ++i) { ms[i] = c->stage_ms[i]; launches[i] = c->stage_launches[i]; }
   return HACK_OK;
 }
 

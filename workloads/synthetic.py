@@ -80,8 +80,9 @@ def _hash_u64(key: int, counter: torch.Tensor) -> torch.Tensor:
 class SyntheticQKV:
     """Generator of per-(layer, scale) Q, K, V for one workload."""
 
-    def __init__(self, cfg: WorkloadConfig, device: str | torch.device = "cpu"):
+    def __init__(self, cfg: WorkloadConfig, device: str | torch.device = "cpu", seed_offset: int = 0):
         self.cfg = cfg
+        self.seed = cfg.seed + 7919 * seed_offset      # the head mask does not depend on the offset
         self.device = torch.device(device)
         self.tokens = cfg.tokens_per_scale
         self.starts = [0]
@@ -128,13 +129,13 @@ class SyntheticQKV:
         t = torch.arange(t0, t0 + n_k, dtype=torch.int64, device=dev).view(1, 1, -1, 1)
         d = torch.arange(c.head_dim, dtype=torch.int64, device=dev).view(1, 1, 1, -1)
         counter = ((b * c.n_heads + h) * self.total + t) * c.head_dim + d
-        return _normal(stream_key(c.seed + layer, layer, tensor), counter)
+        return _normal(stream_key(self.seed + layer, layer, tensor), counter)
 
     def _sink_direction(self, layer: int) -> torch.Tensor:
         """Unit vector u_{l,h} per head, [H, D] fp64 (shared over batch and scales)."""
         c = self.cfg
         idx = torch.arange(c.n_heads * c.head_dim, dtype=torch.int64, device=self.device)
-        g = _normal(stream_key(c.seed + layer, layer, _TENSOR_U), idx).view(c.n_heads, c.head_dim)
+        g = _normal(stream_key(self.seed + layer, layer, _TENSOR_U), idx).view(c.n_heads, c.head_dim)
         return g / torch.linalg.vector_norm(g, dim=1, keepdim=True)
 
     def sink_positions(self, layer: int, scale: int) -> torch.Tensor:
@@ -143,7 +144,7 @@ class SyntheticQKV:
         n_k = self.tokens[scale]
         n_sink = max(1, int(round(c.sink_frac * n_k)))
         idx = torch.arange(c.n_heads * n_k, dtype=torch.int64, device=self.device)
-        hsh = _hash_u64(stream_key(c.seed + layer, layer, _TENSOR_SINK, scale), idx).view(c.n_heads, n_k)
+        hsh = _hash_u64(stream_key(self.seed + layer, layer, _TENSOR_SINK, scale), idx).view(c.n_heads, n_k)
         order = torch.argsort(hsh, dim=1, stable=True)
         flag = torch.zeros(c.n_heads, n_k, dtype=torch.bool, device=self.device)
         flag.scatter_(1, order[:, :n_sink], True)

@@ -152,6 +152,27 @@ HACK_API hack_status_t hack_attend(hack_cache_t* cache, int32_t layer, int32_t s
 HACK_API hack_status_t hack_scale_step(hack_cache_t* cache, int32_t layer, int32_t scale, const void* q,
                               const void* k, const void* v, void* out, void* stream);
 
+/* Scores without any allocation (the paper has no counterpart: this exists for deployment).
+ * For callers that cannot allocate device memory when they need scores - a server whose pool
+ * already owns all of HBM, so cudaMalloc would fail, or a decode loop that cannot afford the
+ * device-wide synchronisation cudaMalloc/cudaFree imply - and therefore cannot create a cache.
+ * Computes what hack_score computes, on dense caller-owned device tensors:
+ *   q       [n_rows, n_queries, head_dim]   (n_rows = batch*heads, dtype as given)
+ *   k_cand  [n_rows, n_cand, head_dim]      all candidate keys of each row, in candidate order
+ *   scores  [n_rows, score_stride] fp32, score_stride >= n_cand; columns j < n_cand are written.
+ * sm_scale 0 selects 1/sqrt(head_dim).  Runs on the calling thread's current device.
+ * Intermediates live in a fixed array inside the library's device image (about 8.3 MiB, held
+ * by every GPU that loads the library until the process exits), hence the limits
+ * n_rows <= 512 and n_rows*n_cand <= 65536; larger sizes return HACK_ERR_UNSUPPORTED.
+ * No cudaMalloc, cudaFree or other allocating call is made.  The first call on a device resolves
+ * the array's address (cudaGetSymbolAddress); make that first call before any stream capture.
+ * All calls share the array: calls that overlap on the GPU race, so keep them on one stream or
+ * order them yourself.  Only enqueues; does not synchronise. */
+HACK_API hack_status_t hack_score_noalloc(const void* q, const void* k_cand, float* scores,
+                                          int32_t n_rows, int32_t n_queries, int32_t n_cand,
+                                          int32_t score_stride, int32_t head_dim, int32_t dtype,
+                                          int32_t n_obs, float sm_scale, void* stream);
+
 /* Same step with HOST buffers (pinned memory recommended): copies Q/K/V to library-owned device
  * staging, runs the step, copies O back, all on `stream`, and returns without synchronising.
  * The staging buffers are allocated by the first such call on a cache. */

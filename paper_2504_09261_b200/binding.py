@@ -21,7 +21,7 @@ RULE_FRACTION, RULE_RATIO = 0, 1
 EXPORTS = (
     "hack_split_budget", "hack_init_cache", "hack_free_cache", "hack_reset", "hack_get_limits",
     "hack_step_info", "hack_score", "hack_select", "hack_compact", "hack_attend", "hack_scale_step",
-    "hack_scale_step_host", "hack_get_lengths", "hack_read_head", "hack_kv_bytes",
+    "hack_scale_step_host", "hack_score_noalloc", "hack_get_lengths", "hack_read_head", "hack_kv_bytes",
     "hack_launch_count", "hack_stage_timing", "hack_stage_times", "hack_poll_status", "hack_last_error",
 )
 
@@ -74,6 +74,7 @@ def _load() -> C.CDLL:
         "hack_attend": [vp, i32, i32, vp, vp, vp],
         "hack_scale_step": [vp, i32, i32, vp, vp, vp, vp, vp],
         "hack_scale_step_host": [vp, i32, i32, vp, vp, vp, vp, vp],
+        "hack_score_noalloc": [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, C.c_float, vp],
         "hack_get_lengths": [vp, i32, C.POINTER(i32)],
         "hack_read_head": [vp, i32, i32, i32, i32, vp, C.c_size_t],
         "hack_kv_bytes": [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)],
@@ -105,6 +106,13 @@ def hack_split_budget(budget: int, alpha: float, rule: int, param: float, total_
     bc, bs = C.c_int32(), C.c_int32()
     _check(lib.hack_split_budget(budget, alpha, rule, param, total_tokens, C.byref(bc), C.byref(bs)))
     return bc.value, bs.value
+
+
+def hack_score_noalloc(q, k_cand, scores, n_rows: int, n_queries: int, n_cand: int, score_stride: int,
+                       head_dim: int, dtype: int, n_obs: int = 32, sm_scale: float = 0.0, stream=None):
+    """Scores on dense device tensors with no device allocation (fixed in-library scratch)."""
+    _check(lib.hack_score_noalloc(_ptr(q), _ptr(k_cand), _ptr(scores), n_rows, n_queries, n_cand,
+                                  score_stride, head_dim, dtype, n_obs, sm_scale, _ptr(stream)))
 
 
 def _ptr(x) -> Optional[int]:

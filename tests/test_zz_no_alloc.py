@@ -1,0 +1,96 @@
+"""hack_score_noalloc against hack_score.
+
+The no-allocation entry point serves callers that cannot create a cache because they cannot
+allocate device memory at that point (all of HBM already belongs to their own pool, or they
+cannot tolerate the device-wide synchronisation an allocation implies).  It must give the same
+scores as the cache-based entry point.  Two calls in a row share the library's fixed scratch, so
+the second call also shows that stale contents of the first do no harm.  Collected last so that
+a failure here cannot hide the result of any other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from workloads import SyntheticQKV, get_config
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    import __graft_entry__ as ge
+    ge.build()
+
+
+def _reference_scores(cfg, layer, upto_scale):
+    """Scores of step `upto_scale` from hack_score on a cache that has not evicted anything yet
+    (tiny budget trigger is avoided by a budget just below the candidate count), together with
+    the dense candidate keys of every (batch, head) row."""
+    import paper_2504_09261_b200 as hb
+    gen = SyntheticQKV(cfg)
+    mask = gen.head_is_contextual.numpy()
+    t_before = sum(cfg.tokens_per_scale[:upto_scale])
+    cand = t_before + cfg.tokens_per_scale[upto_scale]
+    # budgets: nothing is evicted before `upto_scale`, every head is triggered at `upto_scale`
+    budget = cand - 1
+    dtype_id = hb.HACK_F32 if cfg.dtype == "f32" else hb.HACK_BF16
+    cache = hb.HackCache(cfg.n_layers, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides, dtype_id, mask,
+                         budget, budget, n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales)
+    keys = []
+    for k in range(upto_scale):
+        q, kk, v = (t.cuda() for t in gen.qkv(layer, k))
+        out = torch.empty_like(q)
+        cache.hack_scale_step(layer, k, q, kk, v, out)
+        keys.append(kk)
+    q, kk, v = (t.cuda() for t in gen.qkv(layer, upto_scale))
+    keys.append(kk)
+    bh = cfg.batch * cfg.n_heads
+    scores = torch.full((bh, cache.cand_stride), float("nan"), dtype=torch.float32, device="cuda")
+    info = cache.hack_step_info(layer, upto_scale)
+    assert info.triggered_c and info.triggered_s and info.cand_c == cand and info.cand_s == cand
+    cache.hack_score(layer, upto_scale, q, kk, scores)
+    torch.cuda.synchronize()
+    dense_k = torch.cat(keys, dim=2).reshape(bh, cand, cfg.head_dim).contiguous()
+    dense_q = q.reshape(bh, -1, cfg.head_dim).contiguous()
+    ref = scores[:, :cand].clone()
+    cache.close()
+    return dense_q, dense_k, ref, cand, dtype_id
+
+
+@pytest.mark.parametrize("index,scale", [(0, 7), (1, 5)])
+def test_noalloc_scores_match_cache_scores_on_two_calls(index, scale):
+    import paper_2504_09261_b200 as hb
+    cfg = get_config(index, n_layers=1)
+    dense_q, dense_k, ref, cand, dtype_id = _reference_scores(cfg, 0, scale)
+    bh = cfg.batch * cfg.n_heads
+    n_q = dense_q.shape[1]
+    for call in range(2):
+        out = torch.full((bh, cand + 3), float("nan"), dtype=torch.float32, device="cuda")
+        hb.hack_score_noalloc(dense_q, dense_k, out, bh, n_q, cand, cand + 3, cfg.head_dim, dtype_id,
+                              n_obs=cfg.n_obs)
+        torch.cuda.synchronize()
+        got = out[:, :cand]
+        assert torch.isfinite(got).all()
+        assert torch.isnan(out[:, cand:]).all()                       # nothing written past n_cand
+        den = 1e-4 * torch.maximum(got.abs(), ref.abs()) + 1e-7       # the tolerance of the parity tests
+        assert bool(((got - ref).abs() <= den).all()), f"call {call}: max err {(got - ref).abs().max()}"
+        assert abs(float(got.sum(dim=1).mean()) - min(cfg.n_obs, n_q)) < 1e-3
+        if call == 0:
+            # disturb the shared scratch with a different, smaller problem between the two calls
+            small = torch.empty((2, 40), dtype=torch.float32, device="cuda")
+            hb.hack_score_noalloc(dense_q[:2], dense_k[:2, :40].contiguous(), small, 2, n_q, 40, 40,
+                                  cfg.head_dim, dtype_id, n_obs=cfg.n_obs)
+
+
+def test_noalloc_rejects_sizes_beyond_the_fixed_scratch():
+    import paper_2504_09261_b200 as hb
+    q = torch.zeros((1, 1, 64), dtype=torch.float32, device="cuda")
+    with pytest.raises(hb.HackError) as e:
+        hb.hack_score_noalloc(q, q, q, 600, 1, 10, 10, 64, hb.HACK_F32)
+    assert e.value.status == 2 and "scratch" in str(e.value)
+    with pytest.raises(hb.HackError) as e:
+        hb.hack_score_noalloc(q, q, q, 64, 1, 2048, 2048, 64, hb.HACK_F32)
+    assert e.value.status == 2
+    with pytest.raises(hb.HackError) as e:
+        hb.hack_score_noalloc(q, None, q, 1, 1, 1, 1, 64, hb.HACK_F32)
+    assert e.value.status == 1

@@ -1,0 +1,402 @@
+// Attention over the compacted per-head cache on the 5th-generation tensor cores (bf16 inputs,
+// fp32 accumulation): O = Softmax(sm_scale * Q K^T) V with ragged per-head lengths (Eq. 4 on the
+// compressed cache).
+//
+// One CTA serves one (batch, head) and up to two 128-row query tiles, which take turns on the
+// tensor pipe so that the softmax of one tile overlaps the MMAs of the other.
+//   warps 0-3 : softmax of tile 0 (thread r owns query row r: one TMEM lane, no shuffles)
+//   warps 4-7 : softmax of tile 1
+//   warp  8   : TMA producer (Q tiles once, then K and V tiles of 128 cache rows through rings)
+//   warp  9   : tcgen05.mma issuer; also owns the TMEM allocation
+// TMEM (512 columns): S0 [0,128)  S1 [128,256)  O0 [256,256+D)  O1 [256+D,256+2D); the bf16
+// probabilities P_t overwrite the first 64 columns of S_t and feed the second MMA straight from
+// TMEM.  K tiles are K-major operands, V tiles MN-major operands, both 128-byte swizzled as TMA
+// writes them.  Softmax keeps a running maximum that is only raised (and O rescaled in TMEM) when
+// a row's maximum grows by more than 2^8, so rescaling is rare after the first tile.
+// Every mbarrier wait is bounded; on expiry the CTA raises the status word, drains what it has in
+// flight, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "hack_internal.h"
+#include "tc_ptx.cuh"
+
+namespace hack {
+namespace {
+
+using namespace ptx;
+
+constexpr int kBM = 128;                 // query rows per tile
+constexpr int kBN = 128;                 // cache rows per K/V tile
+constexpr int kThreadsTc = 320;
+constexpr int kKStages = 2;
+constexpr int kVStages = 2;
+constexpr uint32_t kSpinLimit = 1u << 22;          // polls while draining after an abort
+constexpr long long kWaitCycles = 2000000000ll;    // about one second: no wait here is legitimately longer
+constexpr float kRescaleThreshold = 8.0f;    // log2 units
+
+struct TcParams {
+  int n_heads, n_new, n_pairs;
+  int kept[2];
+  float scale_log2;                      // sm_scale * log2(e)
+  const uint8_t* is_ctx;
+  const int32_t* row_off;
+  const int32_t* head_order;             // longest heads first
+  __nv_bfloat16* out;
+  int* status;
+};
+
+struct Bars {
+  uint64_t q_full[2];
+  uint64_t k_full[kKStages], k_empty[kKStages];
+  uint64_t v_full[kVStages], v_empty[kVStages];
+  uint64_t s_full[2], p_full[2], o_final[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Bars* b, int* status, int code) {
+  const uint32_t addr = smem_u32(bar);
+  const long long t0 = clock64();
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(addr, parity)) return true;
+    if ((it & 63u) == 63u) {
+      if (*reinterpret_cast<volatile int*>(&b->abort_flag)) return false;
+      if (clock64() - t0 > kWaitCycles) break;
+    }
+  }
+  *reinterpret_cast<volatile int*>(&b->abort_flag) = 1;
+  atomicExch(status, code);
+  return false;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreadsTc, 1)
+attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                 const __grid_constant__ CUtensorMap tm_v, const TcParams p) {
+  constexpr int SUB = D / 64;                       // 64-column (128-byte) sub-tiles per row
+  constexpr uint32_t SUB_BYTES = kBN * 128;         // one sub-tile: 128 rows x 128 bytes
+  constexpr uint32_t TILE_BYTES = SUB * SUB_BYTES;
+  constexpr uint32_t S_COL = 0, O_COL = 256;
+
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t raw = smem_u32(smem_dyn);
+  const uint32_t base = (raw + 1023u) & ~1023u;     // 128-byte swizzle needs 1024-byte alignment
+  unsigned char* sm = smem_dyn + (base - raw);
+  const uint32_t q_sm = base;
+  const uint32_t k_sm = q_sm + 2 * TILE_BYTES;
+  const uint32_t v_sm = k_sm + kKStages * TILE_BYTES;
+  Bars* bars = reinterpret_cast<Bars*>(sm + (2 + kKStages + kVStages) * TILE_BYTES);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bh = p.head_order[blockIdx.x / p.n_pairs];
+  const int pair = blockIdx.x % p.n_pairs;
+  const int len = p.kept[p.is_ctx[bh % p.n_heads]];
+  const int nblk = (len + kBN - 1) / kBN;
+  const int q0 = pair * 2 * kBM;
+  const int ntile = (q0 + kBM < p.n_new) ? 2 : 1;
+
+  if (tid == 0) {
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(smem_u32(&bars->q_full[t]), 1);
+      mbar_init(smem_u32(&bars->s_full[t]), 1);
+      mbar_init(smem_u32(&bars->p_full[t]), kBM);
+      mbar_init(smem_u32(&bars->o_final[t]), 1);
+    }
+    for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
+    for (int s = 0; s < kVStages; ++s) { mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1); }
+    mbar_init(smem_u32(&bars->drain), 1);
+    bars->abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 9) {
+    tmem_alloc(smem_u32(&bars->tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+
+  if (warp == 8) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      prefetch_tensormap(&tm_q);
+      prefetch_tensormap(&tm_k);
+      prefetch_tensormap(&tm_v);
+      const int qrow = bh * p.n_new + q0;
+      for (int t = 0; t < ntile; ++t) {
+        const uint32_t bar = smem_u32(&bars->q_full[t]);
+        mbar_expect_tx(bar, TILE_BYTES);
+        for (int c = 0; c < SUB; ++c)
+          tma_load_2d(q_sm + t * TILE_BYTES + c * SUB_BYTES, &tm_q, c * 64, qrow + t * kBM, bar);
+      }
+      const int krow = p.row_off[bh];
+      int k_issued = 0, v_issued = 0;
+      bool ok = true;
+      for (int j = 0; j < nblk && ok; ++j) {
+        {
+          const int s = j % kKStages;
+          ok = wait_bar(&bars->k_empty[s], ((j / kKStages) & 1) ^ 1, bars, p.status, 1);
+          if (!ok) break;
+          const uint32_t bar = smem_u32(&bars->k_full[s]);
+          mbar_expect_tx(bar, TILE_BYTES);
+          for (int c = 0; c < SUB; ++c)
+            tma_load_2d(k_sm + s * TILE_BYTES + c * SUB_BYTES, &tm_k, c * 64, krow + j * kBN, bar);
+          ++k_issued;
+        }
+        {
+          const int s = j % kVStages;
+          ok = wait_bar(&bars->v_empty[s], ((j / kVStages) & 1) ^ 1, bars, p.status, 2);
+          if (!ok) break;
+          const uint32_t bar = smem_u32(&bars->v_full[s]);
+          mbar_expect_tx(bar, TILE_BYTES);
+          for (int c = 0; c < SUB; ++c)
+            tma_load_2d(v_sm + s * TILE_BYTES + c * SUB_BYTES, &tm_v, c * 64, krow + j * kBN, bar);
+          ++v_issued;
+        }
+      }
+      if (!ok) {
+        // give the copies already in flight a bounded chance to land before the CTA leaves
+        for (int t = 0; t < ntile; ++t) {
+          const uint32_t bar = smem_u32(&bars->q_full[t]);
+          for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar, 0); ++it) {}
+        }
+        for (int i = max(0, k_issued - kKStages); i < k_issued; ++i) {
+          const uint32_t bar = smem_u32(&bars->k_full[i % kKStages]);
+          for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar, (i / kKStages) & 1); ++it) {}
+        }
+        for (int i = max(0, v_issued - kVStages); i < v_issued; ++i) {
+          const uint32_t bar = smem_u32(&bars->v_full[i % kVStages]);
+          for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar, (i / kVStages) & 1); ++it) {}
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t IDESC_S = idesc_bf16_f32(kBM, kBN, 0);
+      constexpr uint32_t IDESC_PV = idesc_bf16_f32(kBM, D, 1);
+      bool ok = true;
+      auto issue_s = [&](int t, int j) {
+        const uint32_t qa = q_sm + t * TILE_BYTES;
+        const uint32_t ka = k_sm + (j % kKStages) * TILE_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk / 4) * SUB_BYTES + (kk % 4) * 32;
+          mma_ss(tmem + S_COL + t * kBN, smem_desc_sw128(qa + off, 16, 1024),
+                 smem_desc_sw128(ka + off, 16, 1024), IDESC_S, kk > 0);
+        }
+        mma_commit(smem_u32(&bars->s_full[t]));
+      };
+      for (int t = 0; t < ntile && ok; ++t) ok = wait_bar(&bars->q_full[t], 0, bars, p.status, 3);
+      if (ok) ok = wait_bar(&bars->k_full[0], 0, bars, p.status, 4);
+      if (ok) {
+        tc_fence_after();
+        for (int t = 0; t < ntile; ++t) issue_s(t, 0);
+        mma_commit(smem_u32(&bars->k_empty[0]));
+      }
+      for (int j = 0; j < nblk && ok; ++j) {
+        const int vs = j % kVStages;
+        for (int t = 0; t < ntile && ok; ++t) {
+          ok = wait_bar(&bars->p_full[t], j & 1, bars, p.status, 5);
+          if (ok && t == 0) ok = wait_bar(&bars->v_full[vs], (j / kVStages) & 1, bars, p.status, 6);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t va = v_sm + vs * TILE_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < kBN / 16; ++kk) {
+            mma_ts(tmem + O_COL + t * D, tmem + S_COL + t * kBN + kk * 8,
+                   smem_desc_sw128(va + kk * 2048, SUB_BYTES, 1024), IDESC_PV, (j > 0 || kk > 0));
+          }
+          if (t == ntile - 1) mma_commit(smem_u32(&bars->v_empty[vs]));
+          if (j + 1 < nblk) {
+            if (t == 0) {
+              ok = wait_bar(&bars->k_full[(j + 1) % kKStages], ((j + 1) / kKStages) & 1, bars, p.status, 7);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            issue_s(t, j + 1);
+            if (t == ntile - 1) mma_commit(smem_u32(&bars->k_empty[(j + 1) % kKStages]));
+          } else {
+            mma_commit(smem_u32(&bars->o_final[t]));
+          }
+        }
+      }
+      if (!ok) {
+        mma_commit(smem_u32(&bars->drain));
+        const uint32_t bar = smem_u32(&bars->drain);
+        for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar, 0); ++it) {}
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue
+    const int t = warp >> 2;                       // tile served by this warpgroup
+    if (t < ntile) {
+      const int r = tid & 127;                     // query row inside the tile == TMEM lane
+      const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+      const uint32_t s_addr = tmem + lane_addr + S_COL + t * kBN;
+      const uint32_t o_addr = tmem + lane_addr + O_COL + t * D;
+      const float c = p.scale_log2;
+      float m_used = -INFINITY, l = 0.f;
+      bool ok = true;
+      for (int j = 0; j < nblk; ++j) {
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[t], j & 1, bars, p.status, 8));
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t sr[kBN];
+#pragma unroll
+        for (int ch = 0; ch < kBN / 32; ++ch) tmem_ld32(s_addr + ch * 32, sr + ch * 32);
+        tmem_wait_ld();
+        const int valid = len - j * kBN;           // >= 1; < 128 only in the last tile
+        if (valid < kBN) {
+#pragma unroll
+          for (int i = 0; i < kBN; ++i)
+            if (i >= valid) sr[i] = 0xff800000u;   // -inf
+        }
+        float mx = __uint_as_float(sr[0]);
+#pragma unroll
+        for (int i = 1; i < kBN; ++i) mx = fmaxf(mx, __uint_as_float(sr[i]));
+        const bool grow = (mx - m_used) * c > kRescaleThreshold;     // always true in the first tile
+        if (__any_sync(0xffffffffu, grow)) {
+          const float m_new = grow ? mx : m_used;
+          const float alpha = grow ? ex2((m_used - m_new) * c) : 1.f;
+          l *= alpha;
+          m_used = m_new;
+          if (j > 0) {
+            // the S_full arrival of this tile also covers the previous P*V MMA, so O is stable
+#pragma unroll
+            for (int ch = 0; ch < D / 32; ++ch) {
+              uint32_t orr[32];
+              tmem_ld32(o_addr + ch * 32, orr);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+              tmem_st32(o_addr + ch * 32, orr);
+            }
+          }
+        }
+        const float mc = m_used * c;
+        float sum = 0.f;
+        uint32_t pk[kBN / 2];
+#pragma unroll
+        for (int i = 0; i < kBN / 2; ++i) {
+          const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), c, -mc));
+          const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), c, -mc));
+          sum += p0 + p1;
+          const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+          pk[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        l += sum;
+        tmem_st32(s_addr, pk);
+        tmem_st32(s_addr + 32, pk + 32);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&bars->p_full[t]));
+      }
+      if (ok) ok = __all_sync(0xffffffffu, wait_bar(&bars->o_final[t], 0, bars, p.status, 9));
+      if (ok) {
+        tc_fence_after();
+        const int row = q0 + t * kBM + r;
+        const float inv = 1.f / l;
+        __nv_bfloat16* dst = p.out + (static_cast<size_t>(bh) * p.n_new + row) * D;
+#pragma unroll
+        for (int ch = 0; ch < D / 32; ++ch) {
+          uint32_t orr[32];
+          tmem_ld32(o_addr + ch * 32, orr);
+          tmem_wait_ld();
+          if (row < p.n_new) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(orr[v * 8 + 2 * e]) * inv,
+                                                               __uint_as_float(orr[v * 8 + 2 * e + 1]) * inv);
+                w[e] = *reinterpret_cast<const uint32_t*>(&h);
+              }
+              *reinterpret_cast<uint4*>(dst + ch * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+template <int D>
+size_t tc_smem_bytes() {
+  return 1024 + (2 + kKStages + kVStages) * (size_t)(D / 64) * kBN * 128 + sizeof(Bars) + 64;
+}
+
+}  // namespace
+
+// 2-D bf16 tensor map over `rows` x `head_dim`, box = 128 rows x 64 columns, 128-byte swizzle.
+bool make_rows_map(void* out_map, const void* base, uint64_t rows, int head_dim) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || rows == 0) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)head_dim, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)head_dim * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)kBN};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(static_cast<CUtensorMap*>(out_map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
+                     const void* q, void* out, cudaStream_t st) {
+  CUtensorMap tm_q;
+  if (!make_rows_map(&tm_q, q, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) return -1;
+  TcParams p;
+  p.n_heads = a.n_heads;
+  p.n_new = a.n_new;
+  p.n_pairs = (a.n_new + 2 * kBM - 1) / (2 * kBM);
+  p.kept[0] = a.kept[0];
+  p.kept[1] = a.kept[1];
+  p.scale_log2 = a.sm_scale * 1.4426950408889634f;
+  p.is_ctx = a.is_ctx;
+  p.row_off = a.row_off;
+  p.head_order = head_order;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.status = a.status;
+  const int grid = p.n_pairs * a.batch * a.n_heads;
+  const CUtensorMap& tk = *static_cast<const CUtensorMap*>(k_map);
+  const CUtensorMap& tv = *static_cast<const CUtensorMap*>(v_map);
+  if (a.head_dim == 128) {
+    static bool set = false;
+    if (!set) { cudaFuncSetAttribute(attend_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes<128>()); set = true; }
+    attend_tc_kernel<128><<<grid, kThreadsTc, tc_smem_bytes<128>(), st>>>(tm_q, tk, tv, p);
+  } else {
+    static bool set = false;
+    if (!set) { cudaFuncSetAttribute(attend_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes<128>()); set = true; }
+    // the larger request keeps it at one CTA per SM (the kernel owns all 512 TMEM columns)
+    attend_tc_kernel<64><<<grid, kThreadsTc, tc_smem_bytes<128>(), st>>>(tm_q, tk, tv, p);
+  }
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace hack

@@ -13,9 +13,9 @@ namespace hack {
 static thread_local std::string g_last_error;
 void set_error(const std::string& msg) { g_last_error = msg; }
 
-int launch_attend_simt(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st);
-
 int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st) {
+  if (dtype == HACK_BF16 && a.n_new >= kTcMinQueries && a.k_map)
+    return launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, st);
   return launch_attend_simt(a, dtype, q, out, st);
 }
 
@@ -28,6 +28,8 @@ struct LayerState {
   int phase = 0;          // 0: scale not started; 1: compacted, attention pending
   int len[2] = {0, 0};    // stored length per head type ([0] structural, [1] contextual)
 };
+
+struct alignas(64) TensorMapBox { unsigned char bytes[128]; };
 
 struct hack_cache {
   hack_config_t cfg;
@@ -54,6 +56,8 @@ struct hack_cache {
   int32_t* idx = nullptr;                       // [b*H, kept_stride]
   hack::Scratch scratch{};
   int* status = nullptr;
+  std::vector<TensorMapBox> k_maps, v_maps;     // per layer, bf16 caches only
+  int32_t* head_order = nullptr;                // [L][2][b*H]: [0] structural heads first, [1] contextual first
   unsigned char* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging
   size_t reserved_bytes = 0, peak_bytes = 0;
   uint64_t launches = 0;
@@ -137,6 +141,12 @@ hack::StepArgs make_args(const hack_cache* c, int layer, int scale, const hack_s
   a.v_plane = c->v_all + c->layer_row_base[layer] * row_bytes;
   a.pos_plane = c->pos_all + c->layer_row_base[layer];
   a.status = c->status;
+  if (!c->k_maps.empty()) {
+    a.k_map = &c->k_maps[layer];
+    a.v_map = &c->v_maps[layer];
+    const int bh = c->cfg.batch * c->cfg.n_heads;
+    a.head_order = c->head_order + ((size_t)layer * 2 + (p.kept_c > p.kept_s ? 1 : 0)) * bh;
+  }
   return a;
 }
 
@@ -332,6 +342,31 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
   c->scratch.max_chunks = (c->limits.cand_stride + hack::kScoreChunk - 1) / hack::kScoreChunk;
   HACK_TRY(cudaMalloc(&c->scratch.logits, (size_t)bh * hack::kMaxObs * c->limits.cand_stride * sizeof(float)));
   HACK_TRY(cudaMalloc(&c->scratch.partials, (size_t)bh * c->scratch.max_chunks * hack::kMaxObs * 2 * sizeof(float)));
+  if (cfg->dtype == HACK_BF16) {
+    // tensor maps of every layer's planes and the two head orders of the tensor-core attention
+    c->k_maps.resize(cfg->n_layers);
+    c->v_maps.resize(cfg->n_layers);
+    std::vector<int32_t> order((size_t)cfg->n_layers * 2 * bh);
+    for (int l = 0; l < cfg->n_layers; ++l) {
+      const size_t rows = c->layer_rows[l] + (l + 1 == cfg->n_layers ? pad_rows : 0);
+      if (!hack::make_rows_map(&c->k_maps[l], c->k_all + c->layer_row_base[l] * row_bytes, rows, cfg->head_dim) ||
+          !hack::make_rows_map(&c->v_maps[l], c->v_all + c->layer_row_base[l] * row_bytes, rows, cfg->head_dim)) {
+        set_error("cuTensorMapEncodeTiled failed for a cache plane");
+        return bail(HACK_ERR_CUDA);
+      }
+      for (int first = 0; first < 2; ++first) {
+        int32_t* o = order.data() + ((size_t)l * 2 + first) * bh;
+        int n = 0;
+        for (int pass = 0; pass < 2; ++pass)
+          for (int i = 0; i < bh; ++i) {
+            const int t = c->mask[(size_t)l * cfg->n_heads + i % cfg->n_heads];
+            if ((pass == 0) == (t == first)) o[n++] = i;
+          }
+      }
+    }
+    HACK_TRY(cudaMalloc(&c->head_order, order.size() * sizeof(int32_t)));
+    HACK_TRY(cudaMemcpy(c->head_order, order.data(), order.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+  }
   HACK_TRY(cudaMalloc(&c->status, sizeof(int)));
   HACK_TRY(cudaMemset(c->status, 0, sizeof(int)));
   HACK_TRY(cudaDeviceSynchronize());
@@ -347,6 +382,7 @@ hack_status_t hack_free_cache(hack_cache_t* c) {
   cudaFree(c->k_all); cudaFree(c->v_all); cudaFree(c->pos_all); cudaFree(c->row_off);
   cudaFree(c->mask_dev); cudaFree(c->scores); cudaFree(c->idx);
   cudaFree(c->scratch.logits); cudaFree(c->scratch.partials); cudaFree(c->status);
+  cudaFree(c->head_order);
   for (int i = 0; i < 4; ++i) cudaFree(c->stage[i]);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   delete c;

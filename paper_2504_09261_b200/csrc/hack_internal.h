@@ -36,6 +36,10 @@ struct StepArgs {
   void* v_plane;
   int32_t* pos_plane;      // device, [rows]
   int* status;             // device status word
+  // tensor-core attention only (host pointers to 128-byte tensor maps of this layer's planes)
+  const void* k_map;
+  const void* v_map;
+  const int32_t* head_order;   // device, [batch*n_heads], heads with the longer cache first
 };
 
 struct Scratch {
@@ -54,6 +58,14 @@ int launch_select(const StepArgs& a, const float* scores, int32_t* idx, int32_t*
 int launch_compact(const StepArgs& a, int dtype, const int32_t* idx, int idx_all, const void* k_new,
                    const void* v_new, cudaStream_t st);
 int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st);
+
+int launch_attend_simt(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st);
+int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
+                     const void* q, void* out, cudaStream_t st);
+// 2-D bf16 tensor map (128 x 64 boxes, 128-byte swizzle) over rows x head_dim; false on failure.
+bool make_rows_map(void* out_map, const void* base, uint64_t rows, int head_dim);
+
+constexpr int kTcMinQueries = 64;   // below this the SIMT kernel serves bf16 as well
 
 void set_error(const std::string& msg);
 

@@ -339,7 +339,7 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
   HACK_TRY(cudaMemcpy(c->mask_dev, c->mask.data(), c->mask.size(), cudaMemcpyHostToDevice));
   HACK_TRY(cudaMalloc(&c->scores, (size_t)bh * c->limits.cand_stride * sizeof(float)));
   HACK_TRY(cudaMalloc(&c->idx, (size_t)bh * c->limits.kept_stride * sizeof(int32_t)));
-  c->scratch.max_chunks = (c->limits.cand_stride + hack::kScoreChunk - 1) / hack::kScoreChunk;
+  c->scratch.max_chunks = c->limits.cand_stride / hack::kScoreChunk + 2;   // stored part and new part are chunked separately
   HACK_TRY(cudaMalloc(&c->scratch.logits, (size_t)bh * hack::kMaxObs * c->limits.cand_stride * sizeof(float)));
   HACK_TRY(cudaMalloc(&c->scratch.partials, (size_t)bh * c->scratch.max_chunks * hack::kMaxObs * 2 * sizeof(float)));
   if (cfg->dtype == HACK_BF16) {

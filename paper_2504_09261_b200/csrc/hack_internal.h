@@ -51,6 +51,9 @@ struct Scratch {
 // Kernel launchers (each returns the number of kernels it enqueued, or -1 on a launch error).
 int launch_score(const StepArgs& a, int dtype, const void* q, const void* k_new, float* scores,
                  const Scratch& s, cudaStream_t st);
+// bf16 caches: the same scores with the logits formed on the tensor cores (two launches).
+int launch_score_tc(const StepArgs& a, const void* q, const void* k_new, float* scores, const Scratch& s,
+                    cudaStream_t st);
 int launch_select(const StepArgs& a, const float* scores, int32_t* idx, int32_t* kept_out,
                   cudaStream_t st);
 // idx == nullptr: every head appends (keeps all candidates).  idx_all != 0: idx rows are valid for

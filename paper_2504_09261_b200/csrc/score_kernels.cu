@@ -195,6 +195,9 @@ int launch_score_t(const StepArgs& a, const void* q, const void* k_new, float* s
 int launch_score(const StepArgs& a, int dtype, const void* q, const void* k_new, float* scores,
                  const Scratch& s, cudaStream_t st) {
   if (!a.trig[0] && !a.trig[1]) return 0;
+  // bf16: tensor-core kernel, unless the new K tensor has fewer rows than one TMA box
+  if (dtype == HACK_BF16 && a.k_map && (long long)a.batch * a.n_heads * a.n_new >= 128)
+    return launch_score_tc(a, q, k_new, scores, s, st);
   if (dtype == HACK_F32) {
     return a.head_dim == 64 ? launch_score_t<float, 64>(a, q, k_new, scores, s, st)
                             : launch_score_t<float, 128>(a, q, k_new, scores, s, st);

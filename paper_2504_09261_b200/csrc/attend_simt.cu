@@ -169,7 +169,7 @@ int launch_attend_simt(const StepArgs& a, int dtype, const void* q, void* out, c
       attend_simt_kernel<__nv_bfloat16, 128><<<grid, kThreads, 0, st>>>(
           a, static_cast<const __nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(out));
   }
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+  return launched(1);
 }
 
 }  // namespace hack

@@ -4,10 +4,22 @@
 //
 // One CTA serves one (batch, head) and up to two 128-row query tiles, which take turns on the
 // tensor pipe so that the softmax of one tile overlaps the MMAs of the other.
-//   warps 0-3 : softmax of tile 0 (thread r owns query row r: one TMEM lane, no shuffles)
-//   warps 4-7 : softmax of tile 1
-//   warp  8   : TMA producer (Q tiles once, then K and V tiles of 128 cache rows through rings)
-//   warp  9   : tcgen05.mma issuer; also owns the TMEM allocation
+//   warp  0     : tcgen05.mma issuer; also owns the TMEM allocation
+//   warp  1     : TMA producer (K and V tiles of 128 cache rows through rings)
+//   warps 4-7   : softmax of tile 0 (thread r owns query row r: one TMEM lane, no shuffles)
+//   warps 8-11  : softmax of tile 1
+//   warps 2-3 only complete the first warpgroup, which hands most of its registers to the
+//   softmax warpgroups (setmaxnreg) so that a whole 128-column score row lives in registers.
+//
+// What shapes the kernel (all measured on the device):
+//  * The thread that issues the MMAs needs instruction-issue slots of its scheduler; many busy
+//    softmax warps starve it (with four always-ready warps per scheduler one tcgen05.mma took
+//    over 200 cycles to issue against about 70 to execute).  Hence one thread per query row (two
+//    softmax warps per scheduler, normally only one of them active) rather than more, lighter
+//    threads, and as few softmax instructions as possible: scale / sum / max work runs on packed
+//    or 3-input instructions.
+//  * Exponentials are scarce (16 per clock and SM against 8192 tensor flops): kPolyOf8 of every
+//    8 pairs are evaluated with a cubic on the FMA pipe instead.
 // TMEM (512 columns): S0 [0,128)  S1 [128,256)  O0 [256,256+D)  O1 [256+D,256+2D); the bf16
 // probabilities P_t overwrite the first 64 columns of S_t and feed the second MMA straight from
 // TMEM.  K tiles are K-major operands, V tiles MN-major operands, both 128-byte swizzled as TMA
@@ -27,7 +39,10 @@ using namespace ptx;
 
 constexpr int kBM = 128;                 // query rows per tile
 constexpr int kBN = 128;                 // cache rows per K/V tile
-constexpr int kThreadsTc = 320;
+constexpr int kThreadsTc = 384;
+constexpr int kMmaWarp = 0, kProducerWarp = 1;   // the issuer is the oldest warp of its scheduler
+constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // 2*128*224 + 128*56 = 384*168 registers
+constexpr int kPolyOf8 = 1;              // pairs out of 8 whose 2^x runs on the FMA pipe
 constexpr int kKStages = 2;
 constexpr int kVStages = 2;
 constexpr uint32_t kSpinLimit = 1u << 22;          // polls while draining after an abort
@@ -57,6 +72,7 @@ struct Bars {
 
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Bars* b, int* status, int code) {
   const uint32_t addr = smem_u32(bar);
+  if (mbar_try_wait(addr, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(addr, parity)) return true;
@@ -100,7 +116,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(&bars->q_full[t]), 1);
       mbar_init(smem_u32(&bars->s_full[t]), 1);
-      mbar_init(smem_u32(&bars->p_full[t]), kBM);
+      mbar_init(smem_u32(&bars->p_full[t]), 4);     // one arrival per warp of the tile
       mbar_init(smem_u32(&bars->o_final[t]), 1);
     }
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
@@ -110,7 +126,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     fence_barrier_init();
     fence_proxy_async();
   }
-  if (warp == 9) {
+  if (warp == kMmaWarp) {
     tmem_alloc(smem_u32(&bars->tmem_base), 512);
     tmem_relinquish();
   }
@@ -119,8 +135,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   tc_fence_after();
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
 
-  if (warp == 8) {
+  if (warp == 2 || warp == 3) {
+    reg_dec<kOtherRegs>();
+  } else if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ TMA producer
+    reg_dec<kOtherRegs>();
     if (lane == 0) {
       prefetch_tensormap(&tm_q);
       prefetch_tensormap(&tm_k);
@@ -173,20 +192,23 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
+    reg_dec<kOtherRegs>();
     if (lane == 0) {
-      constexpr uint32_t IDESC_S = idesc_bf16_f32(kBM, kBN, 0);
-      constexpr uint32_t IDESC_PV = idesc_bf16_f32(kBM, D, 1);
+      constexpr uint32_t IDESC_S = idesc_bf16_f32(kBM, kBN, 0);        // A = Q, B = K (both K-major)
+      constexpr uint32_t IDESC_PV = idesc_bf16_f32(kBM, D, 1);         // A = P (TMEM), B = V (MN-major)
+      // descriptors of the tile bases; a k-step only adds a constant to the address field
+      const uint64_t q_desc[2] = {smem_desc_sw128(q_sm, 16, 1024), smem_desc_sw128(q_sm + TILE_BYTES, 16, 1024)};
+      const uint64_t k_desc0 = smem_desc_sw128(k_sm, 16, 1024);
+      const uint64_t v_desc0 = smem_desc_sw128(v_sm, SUB_BYTES, 1024);
       bool ok = true;
       auto issue_s = [&](int t, int j) {
-        const uint32_t qa = q_sm + t * TILE_BYTES;
-        const uint32_t ka = k_sm + (j % kKStages) * TILE_BYTES;
+        const uint64_t kd = k_desc0 + (uint64_t)(((j % kKStages) * TILE_BYTES) >> 4);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * SUB_BYTES + (kk % 4) * 32;
-          mma_ss(tmem + S_COL + t * kBN, smem_desc_sw128(qa + off, 16, 1024),
-                 smem_desc_sw128(ka + off, 16, 1024), IDESC_S, kk > 0);
+          const uint64_t koff = (uint64_t)(((kk / 4) * SUB_BYTES + (kk % 4) * 32) >> 4);
+          mma_ss(tmem + S_COL + t * kBN, q_desc[t] + koff, kd + koff, IDESC_S, kk > 0);
         }
         mma_commit(smem_u32(&bars->s_full[t]));
       };
@@ -199,17 +221,16 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
       for (int j = 0; j < nblk && ok; ++j) {
         const int vs = j % kVStages;
+        const uint64_t vd = v_desc0 + (uint64_t)((vs * TILE_BYTES) >> 4);
         for (int t = 0; t < ntile && ok; ++t) {
           ok = wait_bar(&bars->p_full[t], j & 1, bars, p.status, 5);
           if (ok && t == 0) ok = wait_bar(&bars->v_full[vs], (j / kVStages) & 1, bars, p.status, 6);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t va = v_sm + vs * TILE_BYTES;
 #pragma unroll
-          for (int kk = 0; kk < kBN / 16; ++kk) {
-            mma_ts(tmem + O_COL + t * D, tmem + S_COL + t * kBN + kk * 8,
-                   smem_desc_sw128(va + kk * 2048, SUB_BYTES, 1024), IDESC_PV, (j > 0 || kk > 0));
-          }
+          for (int kk = 0; kk < kBN / 16; ++kk)
+            mma_ts(tmem + O_COL + t * D, tmem + S_COL + t * kBN + kk * 8, vd + (uint64_t)((kk * 2048) >> 4),
+                   IDESC_PV, (j > 0 || kk > 0));
           if (t == ntile - 1) mma_commit(smem_u32(&bars->v_empty[vs]));
           if (j + 1 < nblk) {
             if (t == 0) {
@@ -232,7 +253,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
-    const int t = warp >> 2;                       // tile served by this warpgroup
+    reg_inc<kSoftmaxRegs>();
+    const int t = (warp >> 2) - 1;                 // tile served by this warpgroup
     if (t < ntile) {
       const int r = tid & 127;                     // query row inside the tile == TMEM lane
       const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -255,9 +277,15 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           for (int i = 0; i < kBN; ++i)
             if (i >= valid) sr[i] = 0xff800000u;   // -inf
         }
-        float mx = __uint_as_float(sr[0]);
+        float mx4[4];
 #pragma unroll
-        for (int i = 1; i < kBN; ++i) mx = fmaxf(mx, __uint_as_float(sr[i]));
+        for (int u = 0; u < 4; ++u) {
+          mx4[u] = fmaxf(__uint_as_float(sr[u * 32]), __uint_as_float(sr[u * 32 + 1]));
+#pragma unroll
+          for (int i = 2; i < 32; i += 2)
+            mx4[u] = max3(mx4[u], __uint_as_float(sr[u * 32 + i]), __uint_as_float(sr[u * 32 + i + 1]));
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         const bool grow = (mx - m_used) * c > kRescaleThreshold;     // always true in the first tile
         if (__any_sync(0xffffffffu, grow)) {
           const float m_new = grow ? mx : m_used;
@@ -266,34 +294,43 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           m_used = m_new;
           if (j > 0) {
             // the S_full arrival of this tile also covers the previous P*V MMA, so O is stable
-#pragma unroll
-            for (int ch = 0; ch < D / 32; ++ch) {
-              uint32_t orr[32];
-              tmem_ld32(o_addr + ch * 32, orr);
+#pragma unroll 1
+            for (int ch = 0; ch < D / 8; ++ch) {             // rare path: kept light on registers
+              uint32_t orr[8];
+              tmem_ld8(o_addr + ch * 8, orr);
               tmem_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
-              tmem_st32(o_addr + ch * 32, orr);
+              for (int i = 0; i < 8; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+              tmem_st8(o_addr + ch * 8, orr);
             }
           }
         }
-        const float mc = m_used * c;
-        float sum = 0.f;
+        const float2 c2 = make_float2(c, c);
+        const float2 nmc2 = make_float2(-m_used * c, -m_used * c);
+        float2 sum4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
         uint32_t pk[kBN / 2];
 #pragma unroll
         for (int i = 0; i < kBN / 2; ++i) {
-          const float p0 = ex2(fmaf(__uint_as_float(sr[2 * i]), c, -mc));
-          const float p1 = ex2(fmaf(__uint_as_float(sr[2 * i + 1]), c, -mc));
-          sum += p0 + p1;
-          const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-          pk[i] = *reinterpret_cast<const uint32_t*>(&h);
+          const float2 x = fma2(make_float2(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1])), c2, nmc2);
+          float2 pr;
+          if ((i & 7) < kPolyOf8) {
+            pr = ex2_poly2(x);
+          } else {
+            pr.x = ex2(x.x);
+            pr.y = ex2(x.y);
+          }
+          sum4[i & 3] = add2(sum4[i & 3], pr);
+          const __nv_bfloat162 hh = __floats2bfloat162_rn(pr.x, pr.y);
+          pk[i] = *reinterpret_cast<const uint32_t*>(&hh);
+          if (i == kBN / 4 - 1) tmem_st32(s_addr, pk);
         }
-        l += sum;
-        tmem_st32(s_addr, pk);
+        const float2 sum2 = add2(add2(sum4[0], sum4[1]), add2(sum4[2], sum4[3]));
+        l += sum2.x + sum2.y;
         tmem_st32(s_addr + 32, pk + 32);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(smem_u32(&bars->p_full[t]));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t]));
       }
       if (ok) ok = __all_sync(0xffffffffu, wait_bar(&bars->o_final[t], 0, bars, p.status, 9));
       if (ok) {
@@ -312,9 +349,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               uint32_t w[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(orr[v * 8 + 2 * e]) * inv,
-                                                               __uint_as_float(orr[v * 8 + 2 * e + 1]) * inv);
-                w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                const __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(orr[v * 8 + 2 * e]) * inv,
+                                                                __uint_as_float(orr[v * 8 + 2 * e + 1]) * inv);
+                w[e] = *reinterpret_cast<const uint32_t*>(&hh);
               }
               *reinterpret_cast<uint4*>(dst + ch * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
@@ -325,7 +362,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == kMmaWarp) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
@@ -396,7 +433,7 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
     // the larger request keeps it at one CTA per SM (the kernel owns all 512 TMEM columns)
     attend_tc_kernel<64><<<grid, kThreadsTc, tc_smem_bytes<128>(), st>>>(tm_q, tk, tv, p);
   }
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+  return launched(1);
 }
 
 }  // namespace hack

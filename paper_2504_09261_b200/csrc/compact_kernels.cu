@@ -167,7 +167,7 @@ int launch_compact(const StepArgs& a, int dtype, const int32_t* idx, int idx_all
   dim3 grid(n_slices + n_copy, 2, heads);
   compact_kernel<<<grid, kThreads, 0, st>>>(a, idx, idx_all, static_cast<const uint4*>(k_new),
                                             static_cast<const uint4*>(v_new), row_pieces, n_slices);
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+  return launched(1);
 }
 
 }  // namespace hack

@@ -424,7 +424,7 @@ hack_status_t hack_score(hack_cache_t* c, int32_t layer, int32_t scale, const vo
   const hack::StepArgs a = make_args(c, layer, scale, p);
   StageScope ts(c, (cudaStream_t)stream, 0);
   const int n = hack::launch_score(a, c->cfg.dtype, q, k_new, scores, c->scratch, (cudaStream_t)stream);
-  if (n < 0) return fail(HACK_ERR_CUDA, "score launch failed");
+  if (n < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
   ts.done(n);
   c->launches += n;
   return HACK_OK;
@@ -440,7 +440,7 @@ hack_status_t hack_select(hack_cache_t* c, int32_t layer, int32_t scale, const f
   const hack::StepArgs a = make_args(c, layer, scale, p);
   StageScope ts(c, (cudaStream_t)stream, 1);
   const int n = hack::launch_select(a, scores, idx, kept_out, (cudaStream_t)stream);
-  if (n < 0) return fail(HACK_ERR_CUDA, "select launch failed");
+  if (n < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
   ts.done(n);
   c->launches += n;
   return HACK_OK;
@@ -457,7 +457,7 @@ hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const 
   const hack::StepArgs a = make_args(c, layer, scale, p);
   StageScope ts(c, (cudaStream_t)stream, 2);
   const int n = hack::launch_compact(a, c->cfg.dtype, idx, 1, k_new, v_new, (cudaStream_t)stream);
-  if (n < 0) return fail(HACK_ERR_CUDA, "compact launch failed");
+  if (n < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
   ts.done(n);
   c->launches += n;
   advance_after_compact(c, layer, p);
@@ -475,7 +475,7 @@ static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void
   const hack::StepArgs a = make_args(c, layer, scale, p);
   StageScope ts(c, st, 3);
   const int n = hack::launch_attend(a, c->cfg.dtype, q, out, st);
-  if (n < 0) return fail(HACK_ERR_CUDA, "attend launch failed");
+  if (n < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
   ts.done(n);
   c->launches += n;
   ls.phase = 0;
@@ -506,20 +506,20 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
   if (any) {
     {
       StageScope ts(c, st, 0);
-      if ((r = hack::launch_score(a, c->cfg.dtype, q, k, c->scores, c->scratch, st)) < 0) return fail(HACK_ERR_CUDA, "score launch failed");
+      if ((r = hack::launch_score(a, c->cfg.dtype, q, k, c->scores, c->scratch, st)) < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
       ts.done(r);
       n += r;
     }
     {
       StageScope ts(c, st, 1);
-      if ((r = hack::launch_select(a, c->scores, c->idx, nullptr, st)) < 0) return fail(HACK_ERR_CUDA, "select launch failed");
+      if ((r = hack::launch_select(a, c->scores, c->idx, nullptr, st)) < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
       ts.done(r);
       n += r;
     }
   }
   {
     StageScope ts(c, st, 2);
-    if ((r = hack::launch_compact(a, c->cfg.dtype, any ? c->idx : nullptr, any ? 1 : 0, k, v, st)) < 0) return fail(HACK_ERR_CUDA, "compact launch failed");
+    if ((r = hack::launch_compact(a, c->cfg.dtype, any ? c->idx : nullptr, any ? 1 : 0, k, v, st)) < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
     ts.done(r);
     n += r;
   }

@@ -72,4 +72,12 @@ constexpr int kTcMinQueries = 64;   // below this the SIMT kernel serves bf16 as
 
 void set_error(const std::string& msg);
 
+// After a kernel launch: n if it was accepted, else -1 with the CUDA error text recorded.
+inline int launched(int n) {
+  const cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) return n;
+  set_error(std::string("kernel launch: ") + cudaGetErrorString(e));
+  return -1;
+}
+
 }  // namespace hack

@@ -187,7 +187,7 @@ int launch_score_t(const StepArgs& a, const void* q, const void* k_new, float* s
       a, static_cast<const T*>(q), static_cast<const T*>(k_new), s.logits, s.partials, s.max_chunks);
   dim3 g2((max_cand + 255) / 256, bh);
   score_reduce_kernel<<<g2, 256, 0, st>>>(a, s.logits, s.partials, s.max_chunks, scores);
-  return cudaGetLastError() == cudaSuccess ? 2 : -1;
+  return launched(2);
 }
 
 }  // namespace

@@ -329,7 +329,7 @@ int launch_t(const StepArgs& a, const CUtensorMap& tm_cache, const CUtensorMap& 
   const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q);
   score_tc_kernel<D, 1><<<grid, kScoreThreads, smem, st>>>(tm_cache, tm_new, a, qp, s.partials, s.max_chunks, per_cta, scores);
   score_tc_kernel<D, 2><<<grid, kScoreThreads, smem, st>>>(tm_cache, tm_new, a, qp, s.partials, s.max_chunks, per_cta, scores);
-  return cudaGetLastError() == cudaSuccess ? 2 : -1;
+  return launched(2);
 }
 
 }  // namespace

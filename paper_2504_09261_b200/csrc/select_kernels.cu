@@ -234,7 +234,7 @@ int launch_select(const StepArgs& a, const float* scores, int32_t* idx, int32_t*
   else if (per_thread <= 12) select_reg_kernel<12><<<grid, kSelThreads, 0, st>>>(a, scores, idx, kept_out);
   else if (per_thread <= kMaxPerThread) select_reg_kernel<kMaxPerThread><<<grid, kSelThreads, 0, st>>>(a, scores, idx, kept_out);
   else select_kernel<<<grid, kSelThreads, 0, st>>>(a, scores, idx, kept_out);
-  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+  return launched(1);
 }
 
 }  // namespace hack

@@ -48,6 +48,7 @@ template <> struct Cvt<__nv_bfloat16> {
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 attend_simt_kernel(const StepArgs a, const T* __restrict__ q, T* __restrict__ out) {
+  pdl_wait();
   constexpr int DQ = D / 4;                       // dims per thread
   constexpr int VEC = Cvt<T>::kPerVec;
   constexpr int ROWV = D / VEC;
@@ -158,15 +159,15 @@ int launch_attend_simt(const StepArgs& a, int dtype, const void* q, void* out, c
   dim3 grid((a.n_new + kQPerCta - 1) / kQPerCta, a.batch * a.n_heads);
   if (dtype == HACK_F32) {
     if (a.head_dim == 64)
-      attend_simt_kernel<float, 64><<<grid, kThreads, 0, st>>>(a, static_cast<const float*>(q), static_cast<float*>(out));
+      launch_k(attend_simt_kernel<float, 64>, grid, kThreads, 0, st, a, static_cast<const float*>(q), static_cast<float*>(out));
     else
-      attend_simt_kernel<float, 128><<<grid, kThreads, 0, st>>>(a, static_cast<const float*>(q), static_cast<float*>(out));
+      launch_k(attend_simt_kernel<float, 128>, grid, kThreads, 0, st, a, static_cast<const float*>(q), static_cast<float*>(out));
   } else {
     if (a.head_dim == 64)
-      attend_simt_kernel<__nv_bfloat16, 64><<<grid, kThreads, 0, st>>>(
+      launch_k(attend_simt_kernel<__nv_bfloat16, 64>, grid, kThreads, 0, st, 
           a, static_cast<const __nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(out));
     else
-      attend_simt_kernel<__nv_bfloat16, 128><<<grid, kThreads, 0, st>>>(
+      launch_k(attend_simt_kernel<__nv_bfloat16, 128>, grid, kThreads, 0, st, 
           a, static_cast<const __nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(out));
   }
   return launched(1);

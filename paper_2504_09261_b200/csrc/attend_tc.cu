@@ -134,6 +134,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
+  pdl_wait();     // everything above overlaps the tail of the previous kernel
 
   if (warp == 2 || warp == 3) {
     reg_dec<kOtherRegs>();
@@ -426,12 +427,12 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
   if (a.head_dim == 128) {
     static bool set = false;
     if (!set) { cudaFuncSetAttribute(attend_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes<128>()); set = true; }
-    attend_tc_kernel<128><<<grid, kThreadsTc, tc_smem_bytes<128>(), st>>>(tm_q, tk, tv, p);
+    launch_k(attend_tc_kernel<128>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, p);
   } else {
     static bool set = false;
     if (!set) { cudaFuncSetAttribute(attend_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes<128>()); set = true; }
     // the larger request keeps it at one CTA per SM (the kernel owns all 512 TMEM columns)
-    attend_tc_kernel<64><<<grid, kThreadsTc, tc_smem_bytes<128>(), st>>>(tm_q, tk, tv, p);
+    launch_k(attend_tc_kernel<64>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, p);
   }
   return launched(1);
 }

@@ -47,6 +47,7 @@ __global__ void __launch_bounds__(kThreads)
 compact_kernel(const StepArgs a, const int32_t* __restrict__ idx, int idx_all,
                const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, int row_pieces,
                int n_slices) {
+  pdl_wait();
   const int bh = blockIdx.z;
   const int ctx = a.is_ctx[bh % a.n_heads];
   const int stored = a.stored[ctx], n_keep = a.kept[ctx];
@@ -165,7 +166,7 @@ int launch_compact(const StepArgs& a, int dtype, const int32_t* idx, int idx_all
   const int cap = (8 * 148 + 2 * heads - 1) / (2 * heads);
   n_copy = n_copy > cap ? cap : n_copy;
   dim3 grid(n_slices + n_copy, 2, heads);
-  compact_kernel<<<grid, kThreads, 0, st>>>(a, idx, idx_all, static_cast<const uint4*>(k_new),
+  launch_k(compact_kernel, grid, kThreads, 0, st, a, idx, idx_all, static_cast<const uint4*>(k_new),
                                             static_cast<const uint4*>(v_new), row_pieces, n_slices);
   return launched(1);
 }

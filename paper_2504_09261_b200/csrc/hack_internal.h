@@ -72,6 +72,31 @@ constexpr int kTcMinQueries = 64;   // below this the SIMT kernel serves bf16 as
 
 void set_error(const std::string& msg);
 
+// Every kernel of the step is launched with programmatic stream serialisation: its CTAs may start
+// while the previous kernel of the stream drains, and stop at pdl_wait() until that kernel has
+// completed and its writes are visible.  Nothing that another kernel produces or still reads is
+// touched before pdl_wait().
+template <typename... KArgs, typename... Args>
+inline void launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#if defined(__CUDACC__)
+__device__ __forceinline__ void pdl_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+
 // After a kernel launch: n if it was accepted, else -1 with the CUDA error text recorded.
 inline int launched(int n) {
   const cudaError_t e = cudaGetLastError();

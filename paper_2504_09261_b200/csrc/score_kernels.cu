@@ -42,6 +42,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kScoreChunk)
 score_logits_kernel(const StepArgs a, const T* __restrict__ q, const T* __restrict__ k_new,
                     float* __restrict__ logits, float* __restrict__ partials, int max_chunks) {
+  pdl_wait();
   constexpr int VEC = Elem<T>::kPerVec;
   constexpr int ROWV = D / VEC;                 // 16-byte vectors per row
   constexpr int KROW = ROWV + 1;                // padded row stride (in vectors) of the key tile
@@ -139,6 +140,7 @@ score_logits_kernel(const StepArgs a, const T* __restrict__ q, const T* __restri
 __global__ void __launch_bounds__(256)
 score_reduce_kernel(const StepArgs a, const float* __restrict__ logits,
                     const float* __restrict__ partials, int max_chunks, float* __restrict__ scores) {
+  pdl_wait();
   const int bh = blockIdx.y;
   const int ctx = a.is_ctx[bh % a.n_heads];
   if (!a.trig[ctx]) return;
@@ -183,10 +185,10 @@ int launch_score_t(const StepArgs& a, const void* q, const void* k_new, float* s
     attr_set = true;
   }
   dim3 g1((max_cand + kScoreChunk - 1) / kScoreChunk, bh);
-  score_logits_kernel<T, D><<<g1, kScoreChunk, smem, st>>>(
+  launch_k(score_logits_kernel<T, D>, g1, kScoreChunk, smem, st, 
       a, static_cast<const T*>(q), static_cast<const T*>(k_new), s.logits, s.partials, s.max_chunks);
   dim3 g2((max_cand + 255) / 256, bh);
-  score_reduce_kernel<<<g2, 256, 0, st>>>(a, s.logits, s.partials, s.max_chunks, scores);
+  launch_k(score_reduce_kernel, g2, 256, 0, st, a, s.logits, s.partials, s.max_chunks, scores);
   return launched(2);
 }
 

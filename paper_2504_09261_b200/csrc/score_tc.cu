@@ -77,6 +77,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_const
   constexpr uint32_t K_BYTES = SUB * K_SUB_BYTES;
   static_assert(STAGES * K_BYTES >= 2 * kMaxObs * kChunkTc * sizeof(float), "ring is reused for the final fold");
 
+  pdl_wait();      // every CTA waits, so that this grid never completes before its predecessor
   const int bh = blockIdx.y;
   const int ctx = a.is_ctx[bh % a.n_heads];
   if (!a.trig[ctx]) return;
@@ -327,8 +328,8 @@ int launch_t(const StepArgs& a, const CUtensorMap& tm_cache, const CUtensorMap& 
   }
   const dim3 grid(splits, heads);
   const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q);
-  score_tc_kernel<D, 1><<<grid, kScoreThreads, smem, st>>>(tm_cache, tm_new, a, qp, s.partials, s.max_chunks, per_cta, scores);
-  score_tc_kernel<D, 2><<<grid, kScoreThreads, smem, st>>>(tm_cache, tm_new, a, qp, s.partials, s.max_chunks, per_cta, scores);
+  launch_k(score_tc_kernel<D, 1>, grid, kScoreThreads, smem, st, tm_cache, tm_new, a, qp, s.partials, s.max_chunks, per_cta, scores);
+  launch_k(score_tc_kernel<D, 2>, grid, kScoreThreads, smem, st, tm_cache, tm_new, a, qp, s.partials, s.max_chunks, per_cta, scores);
   return launched(2);
 }
 

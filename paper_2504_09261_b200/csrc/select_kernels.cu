@@ -94,6 +94,7 @@ template <int E>
 __global__ void __launch_bounds__(kSelThreads)
 select_reg_kernel(const StepArgs a, const float* __restrict__ scores, int32_t* __restrict__ idx,
                   int32_t* __restrict__ kept_out) {
+  pdl_wait();
   const int bh = blockIdx.x;
   const int ctx = a.is_ctx[bh % a.n_heads];
   const int cand = a.cand[ctx], n_keep = a.kept[ctx];
@@ -165,6 +166,7 @@ select_reg_kernel(const StepArgs a, const float* __restrict__ scores, int32_t* _
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const StepArgs a, const float* __restrict__ scores, int32_t* __restrict__ idx,
               int32_t* __restrict__ kept_out) {
+  pdl_wait();
   const int bh = blockIdx.x;
   const int ctx = a.is_ctx[bh % a.n_heads];
   const int cand = a.cand[ctx], n_keep = a.kept[ctx];
@@ -229,11 +231,11 @@ int launch_select(const StepArgs& a, const float* scores, int32_t* idx, int32_t*
   const int grid = a.batch * a.n_heads;
   const int max_cand = a.cand[0] > a.cand[1] ? a.cand[0] : a.cand[1];
   const int per_thread = (max_cand + kSelThreads - 1) / kSelThreads;
-  if (per_thread <= 4) select_reg_kernel<4><<<grid, kSelThreads, 0, st>>>(a, scores, idx, kept_out);
-  else if (per_thread <= 8) select_reg_kernel<8><<<grid, kSelThreads, 0, st>>>(a, scores, idx, kept_out);
-  else if (per_thread <= 12) select_reg_kernel<12><<<grid, kSelThreads, 0, st>>>(a, scores, idx, kept_out);
-  else if (per_thread <= kMaxPerThread) select_reg_kernel<kMaxPerThread><<<grid, kSelThreads, 0, st>>>(a, scores, idx, kept_out);
-  else select_kernel<<<grid, kSelThreads, 0, st>>>(a, scores, idx, kept_out);
+  if (per_thread <= 4) launch_k(select_reg_kernel<4>, grid, kSelThreads, 0, st, a, scores, idx, kept_out);
+  else if (per_thread <= 8) launch_k(select_reg_kernel<8>, grid, kSelThreads, 0, st, a, scores, idx, kept_out);
+  else if (per_thread <= 12) launch_k(select_reg_kernel<12>, grid, kSelThreads, 0, st, a, scores, idx, kept_out);
+  else if (per_thread <= kMaxPerThread) launch_k(select_reg_kernel<kMaxPerThread>, grid, kSelThreads, 0, st, a, scores, idx, kept_out);
+  else launch_k(select_kernel, grid, kSelThreads, 0, st, a, scores, idx, kept_out);
   return launched(1);
 }
 

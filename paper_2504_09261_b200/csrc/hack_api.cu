@@ -14,7 +14,8 @@ static thread_local std::string g_last_error;
 void set_error(const std::string& msg) { g_last_error = msg; }
 
 int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st) {
-  if (dtype == HACK_BF16 && a.n_new >= kTcMinQueries && a.k_map)
+  // the tensor-core kernel serves bf16 caches once a scale has enough rows for its TMA boxes
+  if (dtype == HACK_BF16 && a.k_map && a.n_new >= kTcMinQueries && (long long)a.batch * a.n_heads * a.n_new >= 128)
     return launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, st);
   return launch_attend_simt(a, dtype, q, out, st);
 }
@@ -503,6 +504,18 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
   const hack::StepArgs a = make_args(c, layer, scale, p);
   const bool any = p.triggered_c || p.triggered_s;
   int n = 0, r;
+  if (!any && p.n_new <= hack::kSmallQueries) {
+    // nothing is evicted and the scale is small: one launch appends and attends
+    StageScope ts(c, st, 3);
+    if ((r = hack::launch_append_attend_small(a, c->cfg.dtype, q, k, v, out, st)) < 0) return HACK_ERR_CUDA;
+    ts.done(r);
+    c->launches += r;
+    advance_after_compact(c, layer, p);
+    LayerState& ls = c->layers[layer];
+    ls.phase = 0;
+    ls.next_scale = scale + 1;
+    return HACK_OK;
+  }
   if (any) {
     {
       StageScope ts(c, st, 0);

@@ -68,7 +68,12 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
 // 2-D bf16 tensor map (128 x 64 boxes, 128-byte swizzle) over rows x head_dim; false on failure.
 bool make_rows_map(void* out_map, const void* base, uint64_t rows, int head_dim);
 
-constexpr int kTcMinQueries = 64;   // below this the SIMT kernel serves bf16 as well
+// Untriggered step with at most kSmallQueries new tokens: append and attention in one SIMT launch.
+int launch_append_attend_small(const StepArgs& a, int dtype, const void* q, const void* k_new,
+                               const void* v_new, void* out, cudaStream_t st);
+constexpr int kSmallQueries = 31;
+
+constexpr int kTcMinQueries = 32;   // below this the SIMT kernel serves bf16 as well
 
 void set_error(const std::string& msg);
 

@@ -107,7 +107,7 @@ def test_state_machine_and_argument_errors():
     assert cache.hack_get_lengths(0) == [1] * cfg.n_heads
     live, peak, reserved = cache.hack_kv_bytes()
     assert live == cfg.n_heads * 1 * cfg.head_dim * 4 * 2 and peak == live and reserved > live
-    assert cache.hack_launch_count() >= 2
+    assert cache.hack_launch_count() >= 1
     cache.hack_reset()
     assert cache.hack_get_lengths(0) == [0] * cfg.n_heads
     cache.hack_scale_step(0, 0, q, k, v, out)

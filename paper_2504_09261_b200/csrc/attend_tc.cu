@@ -24,7 +24,7 @@
 // probabilities P_t overwrite the first 64 columns of S_t and feed the second MMA straight from
 // TMEM.  K tiles are K-major operands, V tiles MN-major operands, both 128-byte swizzled as TMA
 // writes them.  Softmax keeps a running maximum that is only raised (and O rescaled in TMEM) when
-// a row's maximum grows by more than 2^8, so rescaling is rare after the first tile.
+// a row's maximum grows by more than 2^32, so rescaling is rare after the first tile.
 // Every mbarrier wait is bounded; on expiry the CTA raises the status word, drains what it has in
 // flight, frees its TMEM and returns.
 #include <cuda.h>
@@ -42,15 +42,16 @@ constexpr int kBN = 128;                 // cache rows per K/V tile
 constexpr int kThreadsTc = 384;
 constexpr int kMmaWarp = 0, kProducerWarp = 1;   // the issuer is the oldest warp of its scheduler
 constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // 2*128*224 + 128*56 = 384*168 registers
-constexpr int kPolyOf8 = 1;              // pairs out of 8 whose 2^x runs on the FMA pipe
+constexpr int kPolyOf8 = 0;              // pairs out of 8 whose 2^x runs on the FMA pipe
 constexpr int kKStages = 2;
 constexpr int kVStages = 2;
 constexpr uint32_t kSpinLimit = 1u << 22;          // polls while draining after an abort
 constexpr long long kWaitCycles = 2000000000ll;    // about one second: no wait here is legitimately longer
-constexpr float kRescaleThreshold = 8.0f;    // log2 units
+constexpr float kRescaleThreshold = 32.0f;   // log2 units: p <= 2^32, far inside the bf16 / fp32 range
 
 struct TcParams {
-  int n_heads, n_new, n_pairs;
+  int n_heads, n_new, n_pairs;           // n_pairs: CTAs per head
+  int tiles_per_cta;                     // 2, or 1 when the grid would not fill the GPU otherwise
   int kept[2];
   float scale_log2;                      // sm_scale * log2(e)
   const uint8_t* is_ctx;
@@ -109,8 +110,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int pair = blockIdx.x % p.n_pairs;
   const int len = p.kept[p.is_ctx[bh % p.n_heads]];
   const int nblk = (len + kBN - 1) / kBN;
-  const int q0 = pair * 2 * kBM;
-  const int ntile = (q0 + kBM < p.n_new) ? 2 : 1;
+  const int q0 = pair * p.tiles_per_cta * kBM;
+  const int ntile = (p.tiles_per_cta == 2 && q0 + kBM < p.n_new) ? 2 : 1;
 
   if (tid == 0) {
     for (int t = 0; t < 2; ++t) {
@@ -206,11 +207,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       bool ok = true;
       auto issue_s = [&](int t, int j) {
         const uint64_t kd = k_desc0 + (uint64_t)(((j % kKStages) * TILE_BYTES) >> 4);
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint64_t koff = (uint64_t)(((kk / 4) * SUB_BYTES + (kk % 4) * 32) >> 4);
-          mma_ss(tmem + S_COL + t * kBN, q_desc[t] + koff, kd + koff, IDESC_S, kk > 0);
-        }
+        if constexpr (D == 128) mma_ss_chain8(tmem + S_COL + t * kBN, q_desc[t], kd, IDESC_S, 0);
+        else mma_ss_chain4(tmem + S_COL + t * kBN, q_desc[t], kd, IDESC_S, 0);
         mma_commit(smem_u32(&bars->s_full[t]));
       };
       for (int t = 0; t < ntile && ok; ++t) ok = wait_bar(&bars->q_full[t], 0, bars, p.status, 3);
@@ -228,10 +226,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           if (ok && t == 0) ok = wait_bar(&bars->v_full[vs], (j / kVStages) & 1, bars, p.status, 6);
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int kk = 0; kk < kBN / 16; ++kk)
-            mma_ts(tmem + O_COL + t * D, tmem + S_COL + t * kBN + kk * 8, vd + (uint64_t)((kk * 2048) >> 4),
-                   IDESC_PV, (j > 0 || kk > 0));
+          mma_ts_chain8(tmem + O_COL + t * D, tmem + S_COL + t * kBN, vd, IDESC_PV, j > 0);
           if (t == ntile - 1) mma_commit(smem_u32(&bars->v_empty[vs]));
           if (j + 1 < nblk) {
             if (t == 0) {
@@ -412,7 +407,10 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
   TcParams p;
   p.n_heads = a.n_heads;
   p.n_new = a.n_new;
-  p.n_pairs = (a.n_new + 2 * kBM - 1) / (2 * kBM);
+  // one query tile per CTA while that still fits one wave: twice the CTAs, no idle SMs
+  const int n_tiles = (a.n_new + kBM - 1) / kBM;
+  p.tiles_per_cta = n_tiles * a.batch * a.n_heads <= 148 ? 1 : 2;
+  p.n_pairs = (n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
   p.kept[0] = a.kept[0];
   p.kept[1] = a.kept[1];
   p.scale_log2 = a.sm_scale * 1.4426950408889634f;

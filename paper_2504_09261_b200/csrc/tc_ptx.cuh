@@ -118,6 +118,60 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
       ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// Chains of MMAs over consecutive 16-element k-steps in ONE asm statement.  The k-step only
+// moves the address field of a descriptor (units of 16 bytes), so the later steps are formed with
+// immediate adds next to the instructions that use them.  Measured in the attention kernel: the
+// issuing thread needs about a quarter less time per MMA than with one asm statement per MMA.
+// `accumulate` applies to the first step; the others always accumulate.
+#define HACK_MMA_SS_STEP(off)                                                        \
+  "add.u64 da, %1, " #off ";\n\tadd.u64 db, %2, " #off ";\n\t"                        \
+  "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, pt;\n\t"
+// D[tmem] (+)= A[smem] * B[smem], both K-major with 128-byte swizzle: k-steps 0..3 inside the
+// first 64-element sub-tile (32 bytes = 2 units apart); steps 4..7 in the second sub-tile, which
+// lies 16 KiB (1024 units) further for a 128-row tile.
+__device__ __forceinline__ void mma_ss_chain4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                              uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, pt;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 pt, %4, %4;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      HACK_MMA_SS_STEP(2) HACK_MMA_SS_STEP(4) HACK_MMA_SS_STEP(6)
+      "}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_ss_chain8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                              uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, pt;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 pt, %4, %4;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      HACK_MMA_SS_STEP(2) HACK_MMA_SS_STEP(4) HACK_MMA_SS_STEP(6)
+      HACK_MMA_SS_STEP(1024) HACK_MMA_SS_STEP(1026) HACK_MMA_SS_STEP(1028) HACK_MMA_SS_STEP(1030)
+      "}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+#undef HACK_MMA_SS_STEP
+// D[tmem] (+)= A[tmem] * B[smem]: A is bf16 in TMEM (8 columns per k-step), B an MN-major tile
+// whose k-step is 16 rows of 128 bytes (128 units).  Eight steps = 128 keys.
+#define HACK_MMA_TS_STEP(k)                                                          \
+  "add.u32 ta, %1, " #k "*8;\n\tadd.u64 db, %2, " #k "*128;\n\t"                      \
+  "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, pt;\n\t"
+__device__ __forceinline__ void mma_ts_chain8(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                              uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, pt;\n\t.reg .b32 ta;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 pt, %4, %4;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
+      HACK_MMA_TS_STEP(1) HACK_MMA_TS_STEP(2) HACK_MMA_TS_STEP(3) HACK_MMA_TS_STEP(4)
+      HACK_MMA_TS_STEP(5) HACK_MMA_TS_STEP(6) HACK_MMA_TS_STEP(7)
+      "}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+#undef HACK_MMA_TS_STEP
+
 // The mbarrier receives one arrival when every MMA this thread issued so far has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");

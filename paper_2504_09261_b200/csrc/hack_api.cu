@@ -57,6 +57,7 @@ struct hack_cache {
   int32_t* idx = nullptr;                       // [b*H, kept_stride]
   hack::Scratch scratch{};
   int* status = nullptr;
+  int32_t* n_old = nullptr;                     // [b*H] scratch of the compaction kernels
   std::vector<TensorMapBox> k_maps, v_maps;     // per layer, bf16 caches only
   int32_t* head_order = nullptr;                // [L][2][b*H]: [0] structural heads first, [1] contextual first
   unsigned char* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging
@@ -142,6 +143,7 @@ hack::StepArgs make_args(const hack_cache* c, int layer, int scale, const hack_s
   a.v_plane = c->v_all + c->layer_row_base[layer] * row_bytes;
   a.pos_plane = c->pos_all + c->layer_row_base[layer];
   a.status = c->status;
+  a.n_old = c->n_old;
   if (!c->k_maps.empty()) {
     a.k_map = &c->k_maps[layer];
     a.v_map = &c->v_maps[layer];
@@ -368,6 +370,7 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
     HACK_TRY(cudaMalloc(&c->head_order, order.size() * sizeof(int32_t)));
     HACK_TRY(cudaMemcpy(c->head_order, order.data(), order.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
   }
+  HACK_TRY(cudaMalloc(&c->n_old, (size_t)bh * sizeof(int32_t)));
   HACK_TRY(cudaMalloc(&c->status, sizeof(int)));
   HACK_TRY(cudaMemset(c->status, 0, sizeof(int)));
   HACK_TRY(cudaDeviceSynchronize());
@@ -384,6 +387,7 @@ hack_status_t hack_free_cache(hack_cache_t* c) {
   cudaFree(c->mask_dev); cudaFree(c->scores); cudaFree(c->idx);
   cudaFree(c->scratch.logits); cudaFree(c->scratch.partials); cudaFree(c->status);
   cudaFree(c->head_order);
+  cudaFree(c->n_old);
   for (int i = 0; i < 4; ++i) cudaFree(c->stage[i]);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   delete c;

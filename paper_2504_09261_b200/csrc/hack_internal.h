@@ -36,6 +36,7 @@ struct StepArgs {
   void* v_plane;
   int32_t* pos_plane;      // device, [rows]
   int* status;             // device status word
+  int32_t* n_old;          // device, [batch*n_heads]: survivors that were already stored (compaction)
   // tensor-core attention only (host pointers to 128-byte tensor maps of this layer's planes)
   const void* k_map;
   const void* v_map;

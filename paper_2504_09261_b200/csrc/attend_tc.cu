@@ -65,7 +65,7 @@ struct Bars {
   uint64_t q_full[2];
   uint64_t k_full[kKStages], k_empty[kKStages];
   uint64_t v_full[kVStages], v_empty[kVStages];
-  uint64_t s_full[2], p_full[2], o_final[2];
+  uint64_t s_full[2], p_full[2][2], o_final[2];    // p_full[t][half]: P of 64 keys is in TMEM
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
@@ -117,7 +117,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(&bars->q_full[t]), 1);
       mbar_init(smem_u32(&bars->s_full[t]), 1);
-      mbar_init(smem_u32(&bars->p_full[t]), 4);     // one arrival per warp of the tile
+      mbar_init(smem_u32(&bars->p_full[t][0]), 4);  // one arrival per warp of the tile
+      mbar_init(smem_u32(&bars->p_full[t][1]), 4);
       mbar_init(smem_u32(&bars->o_final[t]), 1);
     }
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
@@ -222,11 +223,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const int vs = j % kVStages;
         const uint64_t vd = v_desc0 + (uint64_t)((vs * TILE_BYTES) >> 4);
         for (int t = 0; t < ntile && ok; ++t) {
-          ok = wait_bar(&bars->p_full[t], j & 1, bars, p.status, 5);
+          // the probabilities arrive in two halves of 64 keys, so that the second MMA starts while
+          // the softmax is still working on the second half
+          ok = wait_bar(&bars->p_full[t][0], j & 1, bars, p.status, 5);
           if (ok && t == 0) ok = wait_bar(&bars->v_full[vs], (j / kVStages) & 1, bars, p.status, 6);
           if (!ok) break;
           tc_fence_after();
-          mma_ts_chain8(tmem + O_COL + t * D, tmem + S_COL + t * kBN, vd, IDESC_PV, j > 0);
+          mma_ts_chain4(tmem + O_COL + t * D, tmem + S_COL + t * kBN, vd, IDESC_PV, j > 0);
+          ok = wait_bar(&bars->p_full[t][1], j & 1, bars, p.status, 5);
+          if (!ok) break;
+          tc_fence_after();
+          mma_ts_chain4(tmem + O_COL + t * D, tmem + S_COL + t * kBN + 32, vd + 4 * 128, IDESC_PV, 1);
           if (t == ntile - 1) mma_commit(smem_u32(&bars->v_empty[vs]));
           if (j + 1 < nblk) {
             if (t == 0) {
@@ -318,7 +325,14 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           sum4[i & 3] = add2(sum4[i & 3], pr);
           const __nv_bfloat162 hh = __floats2bfloat162_rn(pr.x, pr.y);
           pk[i] = *reinterpret_cast<const uint32_t*>(&hh);
-          if (i == kBN / 4 - 1) tmem_st32(s_addr, pk);
+          if (i == kBN / 4 - 1) {
+            // first 64 keys: hand them to the second MMA now
+            tmem_st32(s_addr, pk);
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t][0]));
+          }
         }
         const float2 sum2 = add2(add2(sum4[0], sum4[1]), add2(sum4[2], sum4[3]));
         l += sum2.x + sum2.y;
@@ -326,7 +340,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t]));
+        if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t][1]));
       }
       if (ok) ok = __all_sync(0xffffffffu, wait_bar(&bars->o_final[t], 0, bars, p.status, 9));
       if (ok) {

@@ -154,18 +154,18 @@ __device__ __forceinline__ void mma_ss_chain8(uint32_t d_tmem, uint64_t adesc, u
 }
 #undef HACK_MMA_SS_STEP
 // D[tmem] (+)= A[tmem] * B[smem]: A is bf16 in TMEM (8 columns per k-step), B an MN-major tile
-// whose k-step is 16 rows of 128 bytes (128 units).  Eight steps = 128 keys.
+// whose k-step is 16 rows of 128 bytes (128 units).
 #define HACK_MMA_TS_STEP(k)                                                          \
   "add.u32 ta, %1, " #k "*8;\n\tadd.u64 db, %2, " #k "*128;\n\t"                      \
   "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, pt;\n\t"
-__device__ __forceinline__ void mma_ts_chain8(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+// Four k-steps (64 keys) starting at k-step 0 of the operands given.
+__device__ __forceinline__ void mma_ts_chain4(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
                                               uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p, pt;\n\t.reg .b32 ta;\n\t.reg .b64 db;\n\t"
       "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 pt, %4, %4;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
-      HACK_MMA_TS_STEP(1) HACK_MMA_TS_STEP(2) HACK_MMA_TS_STEP(3) HACK_MMA_TS_STEP(4)
-      HACK_MMA_TS_STEP(5) HACK_MMA_TS_STEP(6) HACK_MMA_TS_STEP(7)
+      HACK_MMA_TS_STEP(1) HACK_MMA_TS_STEP(2) HACK_MMA_TS_STEP(3)
       "}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");

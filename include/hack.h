@@ -173,9 +173,13 @@ HACK_API hack_status_t hack_score_noalloc(const void* q, const void* k_cand, flo
                                           int32_t score_stride, int32_t head_dim, int32_t dtype,
                                           int32_t n_obs, float sm_scale, void* stream);
 
-/* Same step with HOST buffers (pinned memory recommended): copies Q/K/V to library-owned device
- * staging, runs the step, copies O back, all on `stream`, and returns without synchronising.
- * The staging buffers are allocated by the first such call on a cache. */
+/* Same step with HOST buffers (pinned memory, or the copies are not asynchronous): Q/K/V go to
+ * library-owned device staging, the step runs on `stream`, O comes back; the call returns without
+ * synchronising, and once `stream` has been synchronised out_host is complete.  The uploads and
+ * the download run on two private streams with three staging sets, so the upload of the next
+ * call overlaps this call's kernels; the host buffers of a call must stay valid until `stream`
+ * has passed that call.  The staging sets and streams are created by the first such call on a
+ * cache (make it outside any stream capture). */
 HACK_API hack_status_t hack_scale_step_host(hack_cache_t* cache, int32_t layer, int32_t scale,
                                    const void* q_host, const void* k_host, const void* v_host,
                                    void* out_host, void* stream);

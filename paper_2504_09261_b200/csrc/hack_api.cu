@@ -60,7 +60,13 @@ struct hack_cache {
   int32_t* n_old = nullptr;                     // [b*H] scratch of the compaction kernels
   std::vector<TensorMapBox> k_maps, v_maps;     // per layer, bf16 caches only
   int32_t* head_order = nullptr;                // [L][2][b*H]: [0] structural heads first, [1] contextual first
-  unsigned char* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging
+  // host-buffer entry point: kHostSlots staging sets (q, k, v, o) cycled call by call, copies on
+  // two private streams so that the next call's upload runs under this call's kernels
+  static constexpr int kHostSlots = 3;
+  unsigned char* stage[kHostSlots][4] = {};
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  cudaEvent_t ev_in[kHostSlots] = {}, ev_step[kHostSlots] = {}, ev_out[kHostSlots] = {};
+  uint64_t host_calls = 0;
   size_t reserved_bytes = 0, peak_bytes = 0;
   uint64_t launches = 0;
   // optional per-stage device timing (score, select, compact, attend)
@@ -388,7 +394,14 @@ hack_status_t hack_free_cache(hack_cache_t* c) {
   cudaFree(c->scratch.logits); cudaFree(c->scratch.partials); cudaFree(c->status);
   cudaFree(c->head_order);
   cudaFree(c->n_old);
-  for (int i = 0; i < 4; ++i) cudaFree(c->stage[i]);
+  for (int sl = 0; sl < hack_cache::kHostSlots; ++sl) {
+    for (int i = 0; i < 4; ++i) cudaFree(c->stage[sl][i]);
+    if (c->ev_in[sl]) cudaEventDestroy(c->ev_in[sl]);
+    if (c->ev_step[sl]) cudaEventDestroy(c->ev_step[sl]);
+    if (c->ev_out[sl]) cudaEventDestroy(c->ev_out[sl]);
+  }
+  if (c->h2d_stream) cudaStreamDestroy(c->h2d_stream);
+  if (c->d2h_stream) cudaStreamDestroy(c->d2h_stream);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   delete c;
   return HACK_OK;
@@ -552,23 +565,48 @@ hack_status_t hack_scale_step_host(hack_cache_t* c, int32_t layer, int32_t scale
   if (!q_host || !k_host || !v_host || !out_host) return fail(HACK_ERR_INVALID_ARG, "a host buffer is NULL");
   cudaStream_t st = (cudaStream_t)stream;
   const size_t full = (size_t)c->cfg.batch * c->cfg.n_heads * c->limits.max_new * c->cfg.head_dim * c->elt;
-  if (!c->stage[0]) {
-    for (int i = 0; i < 4; ++i) {
-      cudaError_t e = cudaMalloc(&c->stage[i], full);
-      if (e != cudaSuccess) {
-        for (int j = 0; j < 4; ++j) { cudaFree(c->stage[j]); c->stage[j] = nullptr; }
-        set_error(std::string("staging cudaMalloc: ") + cudaGetErrorString(e));
-        return HACK_ERR_OOM;
-      }
+  if (!c->h2d_stream) {
+    // first use: staging sets, the two copy streams and the events that order them
+    bool ok = cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int sl = 0; sl < hack_cache::kHostSlots && ok; ++sl) {
+      for (int i = 0; i < 4 && ok; ++i) ok = cudaMalloc(&c->stage[sl][i], full) == cudaSuccess;
+      ok = ok && cudaEventCreateWithFlags(&c->ev_in[sl], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&c->ev_step[sl], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&c->ev_out[sl], cudaEventDisableTiming) == cudaSuccess;
+    }
+    if (!ok) {
+      set_error(std::string("staging set-up: ") + cudaGetErrorString(cudaGetLastError()));
+      for (int sl = 0; sl < hack_cache::kHostSlots; ++sl)
+        for (int i = 0; i < 4; ++i) { cudaFree(c->stage[sl][i]); c->stage[sl][i] = nullptr; }
+      if (c->h2d_stream) { cudaStreamDestroy(c->h2d_stream); c->h2d_stream = nullptr; }
+      if (c->d2h_stream) { cudaStreamDestroy(c->d2h_stream); c->d2h_stream = nullptr; }
+      return HACK_ERR_OOM;
     }
   }
+  const int sl = (int)(c->host_calls % hack_cache::kHostSlots);
+  const bool reused = c->host_calls >= (uint64_t)hack_cache::kHostSlots;
+  unsigned char** sg = c->stage[sl];
   const size_t bytes = (size_t)c->cfg.batch * c->cfg.n_heads * c->n_tok[scale] * c->cfg.head_dim * c->elt;
-  HACK_CUDA(cudaMemcpyAsync(c->stage[0], q_host, bytes, cudaMemcpyHostToDevice, st));
-  HACK_CUDA(cudaMemcpyAsync(c->stage[1], k_host, bytes, cudaMemcpyHostToDevice, st));
-  HACK_CUDA(cudaMemcpyAsync(c->stage[2], v_host, bytes, cudaMemcpyHostToDevice, st));
-  s = hack_scale_step(c, layer, scale, c->stage[0], c->stage[1], c->stage[2], c->stage[3], stream);
+  // upload: after the step that last read this staging set, not after anything else on `stream`
+  if (reused) HACK_CUDA(cudaStreamWaitEvent(c->h2d_stream, c->ev_step[sl], 0));
+  HACK_CUDA(cudaMemcpyAsync(sg[0], q_host, bytes, cudaMemcpyHostToDevice, c->h2d_stream));
+  HACK_CUDA(cudaMemcpyAsync(sg[1], k_host, bytes, cudaMemcpyHostToDevice, c->h2d_stream));
+  HACK_CUDA(cudaMemcpyAsync(sg[2], v_host, bytes, cudaMemcpyHostToDevice, c->h2d_stream));
+  HACK_CUDA(cudaEventRecord(c->ev_in[sl], c->h2d_stream));
+  // the step, on the caller's stream (the output staging buffer is free: the stream waited for
+  // its download at the end of the call that used it)
+  HACK_CUDA(cudaStreamWaitEvent(st, c->ev_in[sl], 0));
+  s = hack_scale_step(c, layer, scale, sg[0], sg[1], sg[2], sg[3], stream);
   if (s != HACK_OK) return s;
-  HACK_CUDA(cudaMemcpyAsync(out_host, c->stage[3], bytes, cudaMemcpyDeviceToHost, st));
+  HACK_CUDA(cudaEventRecord(c->ev_step[sl], st));
+  // download on its own stream; the caller's stream joins it, so that synchronising `stream`
+  // still means out_host is complete
+  HACK_CUDA(cudaStreamWaitEvent(c->d2h_stream, c->ev_step[sl], 0));
+  HACK_CUDA(cudaMemcpyAsync(out_host, sg[3], bytes, cudaMemcpyDeviceToHost, c->d2h_stream));
+  HACK_CUDA(cudaEventRecord(c->ev_out[sl], c->d2h_stream));
+  HACK_CUDA(cudaStreamWaitEvent(st, c->ev_out[sl], 0));
+  ++c->host_calls;
   return HACK_OK;
 }
 

@@ -229,7 +229,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_const
       }
       consumer_sync();
 #pragma unroll
-      for (int i = 0; i < kMaxObs; ++i) { rm[i] = row_m[i]; rl[i] = i < a.n_obs_rows ? row_inv_l[i] : 0.f; }
+      for (int i = 0; i < kMaxObs; ++i) {        // rows past n_obs_rows are padding: weight 0, finite reference
+        rm[i] = i < a.n_obs_rows ? row_m[i] : 0.f;
+        rl[i] = i < a.n_obs_rows ? row_inv_l[i] : 0.f;
+      }
     }
     bool ok = true;
     for (int i = 0; i < n_run; ++i) {

@@ -1,0 +1,120 @@
+"""GPU parity on shapes outside the five benchmark workloads: the code paths that only unusual
+sizes reach (long candidate lists, odd head counts, head_dim 128 in fp32, one observation row,
+a single scale) still have to agree with the CPU oracle under the same teacher-forced protocol."""
+from dataclasses import replace
+
+import pytest
+
+from workloads import get_config
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    import __graft_entry__ as ge
+    ge.build()
+
+
+def _ok(rep):
+    assert rep.ok(), rep.summary() + "\n" + "\n".join(rep.problems)
+    assert rep.heads_checked > 0
+
+
+def _custom(base_index, **kw):
+    cfg = get_config(base_index, n_layers=1)
+    return replace(cfg, name=cfg.name + "-custom", **kw)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_long_candidate_list_takes_the_general_selection_path(dtype):
+    """17 429 candidates per head: more than the register-resident selection holds (16 384), many
+    scoring chunks per head, a ragged last chunk.  The new scale competes (policy 1) so that the
+    kept length stays small and the oracle's attention stays cheap."""
+    from tests.parity_util import run_parity
+    cfg = _custom(0, sides=(1, 2, 132), n_heads=2, batch=1, dtype=dtype)
+    rep = run_parity(cfg, layers=[0], fused=True, budget_c=300, budget_s=500, policy=1)
+    _ok(rep)
+    assert rep.compressed_heads > 0
+
+
+def test_fp32_head_dim_128_and_odd_head_count():
+    """fp32 runs on the SIMT kernels only; head_dim 128 and 3 heads x batch 1 are not in config 0."""
+    from tests.parity_util import run_parity
+    cfg = _custom(0, head_dim=128, n_heads=3, batch=1, sides=(1, 2, 3, 5, 9, 14))
+    rep = run_parity(cfg, layers=[0], fused=True, budget_c=40, budget_s=120)
+    _ok(rep)
+    assert rep.compressed_heads > 0
+
+
+def test_bf16_small_grid_single_query_tile_per_cta():
+    """Few heads and a mid-sized scale: the tensor-core attention runs with one query tile per CTA
+    and ragged last tiles in both the query and the key direction."""
+    from tests.parity_util import run_parity
+    cfg = _custom(3, n_heads=3, batch=1, sides=(1, 2, 4, 7, 11, 19))
+    rep = run_parity(cfg, layers=[0], fused=True, budget_c=90, budget_s=400)
+    _ok(rep)
+    assert rep.compressed_heads > 0
+
+
+def test_single_observation_row_and_single_scale():
+    """n_obs = 1 (one query row scores every key) and a schedule of one scale."""
+    from tests.parity_util import run_parity
+    cfg = _custom(1, n_obs=1, n_heads=4, batch=1, sides=(1, 2, 4, 8, 12))
+    rep = run_parity(cfg, layers=[0], fused=True, budget_c=20, budget_s=100)
+    _ok(rep)
+    one = _custom(1, n_heads=2, batch=1, sides=(9,), n_init_scales=1)
+    rep = run_parity(one, layers=[0], fused=True, budget_c=30, budget_s=50, policy=1)
+    _ok(rep)
+
+
+def test_graph_replay_reproduces_direct_calls():
+    """bench.py times CUDA-graph replays of the hack_scale_step calls; a replay has to write the
+    same bytes as the direct calls did (the length plan is fixed, so a captured loop is complete)."""
+    import torch
+    from workloads import SyntheticQKV
+    import paper_2504_09261_b200 as hb
+    cfg = get_config(1, n_layers=2)
+    dev = torch.device("cuda:0")
+    gen = SyntheticQKV(cfg, device=dev)
+    mask = gen.head_is_contextual
+    L, K = cfg.n_layers, cfg.n_scales
+    qkv = [[gen.qkv(l, k) for k in range(K)] for l in range(L)]
+
+    def fresh():
+        return hb.HackCache(L, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides, hb.HACK_BF16, mask.numpy(),
+                            cfg.budget_c, cfg.budget_s, device=0)
+
+    def loop(cache, outs, stream_handle):
+        cache.hack_reset()
+        for k in range(K):
+            for l in range(L):
+                q, kk, v = qkv[l][k]
+                cache.hack_scale_step(l, k, q, kk, v, outs[l][k], stream_handle)
+
+    direct = fresh()
+    out_a = [[torch.zeros_like(qkv[l][k][0]) for k in range(K)] for l in range(L)]
+    loop(direct, out_a, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+
+    replayed = fresh()
+    out_b = [[torch.zeros_like(qkv[l][k][0]) for k in range(K)] for l in range(L)]
+    loop(replayed, out_b, torch.cuda.current_stream().cuda_stream)     # one-time kernel attributes
+    torch.cuda.synchronize()
+    for row in out_b:
+        for t in row:
+            t.zero_()
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.graph(g, stream=side):
+        loop(replayed, out_b, torch.cuda.current_stream().cuda_stream)
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize()
+    for l in range(L):
+        for k in range(K):
+            assert torch.equal(out_a[l][k].view(torch.int16), out_b[l][k].view(torch.int16)), (l, k)
+    for l in range(L):
+        assert direct.hack_get_lengths(l) == replayed.hack_get_lengths(l)
+    direct.close()
+    replayed.close()

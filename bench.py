@@ -27,6 +27,7 @@ if ROOT not in sys.path:
 import torch  # noqa: E402
 
 from workloads import SyntheticQKV, get_config  # noqa: E402
+from workloads import sharding  # noqa: E402
 
 METRIC = "scale-step tokens/s (score+select+compact+attend)"
 UNIT = "tokens/s"
@@ -202,7 +203,7 @@ def run_ours(args):
     if args.layers:
         cfg = cfg.with_layers(args.layers)
     L, K = cfg.n_layers, cfg.n_scales
-    gen = SyntheticQKV(cfg, device=dev, seed_offset=rank)      # each rank decodes its own images
+    gen = sharding.rank_generator(cfg, rank, device=dev)        # each rank decodes its own images
     mask = gen.head_is_contextual
     n_ctx = [int(mask[l].sum()) for l in range(L)]
     dtype_id = hb.HACK_F32 if cfg.dtype == "f32" else hb.HACK_BF16
@@ -302,13 +303,10 @@ def run_ours(args):
     sampler.start()
     total_ms, scale_ms = timed(cache, args.steps, args.warmup, per_scale=True, use_graph=use_graph)
     clocks = sampler.stop()
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = sharding.max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms / args.steps
     tokens = cfg.batch * cfg.total_tokens
-    value = world * tokens / (ms_per_step * 1e-3)
+    value = sharding.job_throughput(world, tokens, ms_per_step)
     live, peak, reserved = cache.hack_kv_bytes()
 
     # ---- work model and roofline of the loop
@@ -439,11 +437,8 @@ def run_ours(args):
         e1.record(stream)
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / n_e2e
-        if dist is not None:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        e2e = {"value": world * tokens / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+        ms = sharding.max_over_ranks(ms, dist, dev)
+        e2e = {"value": sharding.job_throughput(world, tokens, ms), "unit": UNIT, "ms_per_step": ms,
                "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": in_bytes // 3}
         c2.close()
         del host, host_out

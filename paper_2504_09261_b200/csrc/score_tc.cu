@@ -182,6 +182,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_const
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t IDESC = idesc_bf16_f32(kChunkTc, kMaxObs, 0);
+      const uint64_t q_desc = smem_desc_sw128(q_sm, 16, 1024);
       bool ok = true;
       for (int i = 0; i < n_run && ok; ++i) {
         const int s = i % STAGES, b = i % kAccBufs;
@@ -189,13 +190,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_const
         if (ok) ok = wait_bar(&bars->acc_free[b], ((i / kAccBufs) & 1) ^ 1, bars, a.status, 13);
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t ko = s * K_BYTES + (kk / 4) * K_SUB_BYTES + (kk % 4) * 32;
-          const uint32_t qo = (kk / 4) * Q_SUB_BYTES + (kk % 4) * 32;
-          mma_ss(tmem + b * kMaxObs, smem_desc_sw128(k_sm + ko, 16, 1024), smem_desc_sw128(q_sm + qo, 16, 1024),
-                 IDESC, kk > 0);
-        }
+        const uint64_t k_desc = smem_desc_sw128(k_sm + s * K_BYTES, 16, 1024);
+        if constexpr (D == 128) mma_ss_chain8_b32rows(tmem + b * kMaxObs, k_desc, q_desc, IDESC, 0);
+        else mma_ss_chain4(tmem + b * kMaxObs, k_desc, q_desc, IDESC, 0);
         mma_commit(smem_u32(&bars->empty[s]));
         mma_commit(smem_u32(&bars->acc_full[b]));
       }

@@ -153,6 +153,24 @@ __device__ __forceinline__ void mma_ss_chain8(uint32_t d_tmem, uint64_t adesc, u
       : "memory");
 }
 #undef HACK_MMA_SS_STEP
+// Same chain when the B tile has only 32 rows (its second sub-tile lies 4 KiB = 256 units on).
+#define HACK_MMA_SS_STEP_AB(offa, offb)                                              \
+  "add.u64 da, %1, " #offa ";\n\tadd.u64 db, %2, " #offb ";\n\t"                      \
+  "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, pt;\n\t"
+__device__ __forceinline__ void mma_ss_chain8_b32rows(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                      uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, pt;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 pt, %4, %4;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      HACK_MMA_SS_STEP_AB(2, 2) HACK_MMA_SS_STEP_AB(4, 4) HACK_MMA_SS_STEP_AB(6, 6)
+      HACK_MMA_SS_STEP_AB(1024, 256) HACK_MMA_SS_STEP_AB(1026, 258) HACK_MMA_SS_STEP_AB(1028, 260)
+      HACK_MMA_SS_STEP_AB(1030, 262)
+      "}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+#undef HACK_MMA_SS_STEP_AB
 // D[tmem] (+)= A[tmem] * B[smem]: A is bf16 in TMEM (8 columns per k-step), B an MN-major tile
 // whose k-step is 16 rows of 128 bytes (128 units).
 #define HACK_MMA_TS_STEP(k)                                                          \

@@ -437,12 +437,10 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
   const CUtensorMap& tk = *static_cast<const CUtensorMap*>(k_map);
   const CUtensorMap& tv = *static_cast<const CUtensorMap*>(v_map);
   if (a.head_dim == 128) {
-    static bool set = false;
-    if (!set) { cudaFuncSetAttribute(attend_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes<128>()); set = true; }
+    allow_dynamic_smem(attend_tc_kernel<128>, tc_smem_bytes<128>());
     launch_k(attend_tc_kernel<128>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, p);
   } else {
-    static bool set = false;
-    if (!set) { cudaFuncSetAttribute(attend_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes<128>()); set = true; }
+    allow_dynamic_smem(attend_tc_kernel<64>, tc_smem_bytes<128>());
     // the larger request keeps it at one CTA per SM (the kernel owns all 512 TMEM columns)
     launch_k(attend_tc_kernel<64>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, p);
   }

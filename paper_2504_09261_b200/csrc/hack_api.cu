@@ -4,7 +4,9 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
+#include <utility>
 
 #include "hack_internal.h"
 
@@ -12,6 +14,18 @@ namespace hack {
 
 static thread_local std::string g_last_error;
 void set_error(const std::string& msg) { g_last_error = msg; }
+
+void allow_dynamic_smem_impl(const void* kern, size_t bytes) {
+  static std::mutex mu;
+  static std::vector<std::pair<const void*, int>> done;        // (kernel, device) pairs already served
+  int dev = 0;
+  cudaGetDevice(&dev);
+  std::lock_guard<std::mutex> lock(mu);
+  for (const auto& kd : done)
+    if (kd.first == kern && kd.second == dev) return;
+  cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  done.emplace_back(kern, dev);
+}
 
 int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st) {
   // the tensor-core kernel serves bf16 caches once a scale has enough rows for its TMA boxes

@@ -103,6 +103,14 @@ __device__ __forceinline__ void pdl_wait() {
 }
 #endif
 
+// Opt-in to more than 48 KB of dynamic shared memory.  The attribute belongs to the (function,
+// device) pair, so it is set once per pair, on the device that is current (thread safe).
+void allow_dynamic_smem_impl(const void* kern, size_t bytes);
+template <typename F>
+inline void allow_dynamic_smem(F* kern, size_t bytes) {
+  allow_dynamic_smem_impl(reinterpret_cast<const void*>(kern), bytes);
+}
+
 // After a kernel launch: n if it was accepted, else -1 with the CUDA error text recorded.
 inline int launched(int n) {
   const cudaError_t e = cudaGetLastError();

@@ -320,12 +320,8 @@ int launch_t(const StepArgs& a, const CUtensorMap& tm_cache, const CUtensorMap& 
   if (splits > s.max_chunks) return -1;
   const size_t smem = 1024 + (size_t)STAGES * (D / 64) * kChunkTc * 128 + (size_t)(D / 64) * kMaxObs * 128 +
                       sizeof(ScoreBars) + 16;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(score_tc_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    cudaFuncSetAttribute(score_tc_kernel<D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    attr_set = true;
-  }
+  allow_dynamic_smem(score_tc_kernel<D, 1>, smem);
+  allow_dynamic_smem(score_tc_kernel<D, 2>, smem);
   const dim3 grid(splits, heads);
   const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q);
   launch_k(score_tc_kernel<D, 1>, grid, kScoreThreads, smem, st, tm_cache, tm_new, a, qp, s.partials, s.max_chunks, per_cta, scores);

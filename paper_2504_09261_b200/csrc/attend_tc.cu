@@ -113,7 +113,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int q0 = pair * p.tiles_per_cta * kBM;
   const int ntile = (p.tiles_per_cta == 2 && q0 + kBM < p.n_new) ? 2 : 1;
 
-  if (tid == 0) {
+  const int qrow = bh * p.n_new + q0;
+  const int krow = p.row_off[bh];
+  if (warp == kProducerWarp && lane == 0) {
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(&bars->q_full[t]), 1);
       mbar_init(smem_u32(&bars->s_full[t]), 1);
@@ -127,6 +129,22 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     bars->abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
+    // the producer starts the first loads at once: they run under the TMEM allocation, the
+    // block-wide synchronisation and the register reallocation below
+    prefetch_tensormap(&tm_q);
+    prefetch_tensormap(&tm_k);
+    prefetch_tensormap(&tm_v);
+    pdl_wait();
+    for (int t = 0; t < ntile; ++t) {
+      const uint32_t bar = smem_u32(&bars->q_full[t]);
+      mbar_expect_tx(bar, TILE_BYTES);
+      for (int c = 0; c < SUB; ++c)
+        tma_load_2d(q_sm + t * TILE_BYTES + c * SUB_BYTES, &tm_q, c * 64, qrow + t * kBM, bar);
+    }
+    mbar_expect_tx(smem_u32(&bars->k_full[0]), TILE_BYTES);
+    for (int c = 0; c < SUB; ++c) tma_load_2d(k_sm + c * SUB_BYTES, &tm_k, c * 64, krow, smem_u32(&bars->k_full[0]));
+    mbar_expect_tx(smem_u32(&bars->v_full[0]), TILE_BYTES);
+    for (int c = 0; c < SUB; ++c) tma_load_2d(v_sm + c * SUB_BYTES, &tm_v, c * 64, krow, smem_u32(&bars->v_full[0]));
   }
   if (warp == kMmaWarp) {
     tmem_alloc(smem_u32(&bars->tmem_base), 512);
@@ -144,20 +162,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // ------------------------------------------------------------------ TMA producer
     reg_dec<kOtherRegs>();
     if (lane == 0) {
-      prefetch_tensormap(&tm_q);
-      prefetch_tensormap(&tm_k);
-      prefetch_tensormap(&tm_v);
-      const int qrow = bh * p.n_new + q0;
-      for (int t = 0; t < ntile; ++t) {
-        const uint32_t bar = smem_u32(&bars->q_full[t]);
-        mbar_expect_tx(bar, TILE_BYTES);
-        for (int c = 0; c < SUB; ++c)
-          tma_load_2d(q_sm + t * TILE_BYTES + c * SUB_BYTES, &tm_q, c * 64, qrow + t * kBM, bar);
-      }
-      const int krow = p.row_off[bh];
-      int k_issued = 0, v_issued = 0;
+      int k_issued = 1, v_issued = 1;               // Q and tile 0 of K and V are already on their way
       bool ok = true;
-      for (int j = 0; j < nblk && ok; ++j) {
+      for (int j = 1; j < nblk && ok; ++j) {
         {
           const int s = j % kKStages;
           ok = wait_bar(&bars->k_empty[s], ((j / kKStages) & 1) ^ 1, bars, p.status, 1);

@@ -53,10 +53,30 @@ def split_budget(budget: int, alpha: float, rule: str, param: float, total_token
 
 
 # --------------------------------------------------------------------------- step pieces
-def observation_rows(n_k: int, n_obs: int) -> np.ndarray:
-    """Indices of the uniformly spaced query subset: floor(m * N_k / n), n = min(N_obs, N_k)."""
+UNIFORM, INIT, RECENT, CALLER = 0, 1, 2, 3   # query-subset rules of the sampling ablation (Table "qselect")
+
+
+def observation_rows(n_k: int, n_obs: int, sampler: int = UNIFORM,
+                     caller_rows: Optional[Sequence[int]] = None) -> np.ndarray:
+    """Indices of the query subset Q~ of Eq. 9, n = min(N_obs, N_k) rows of the current scale.
+
+    UNIFORM (the method's rule): floor(m * N_k / n).  INIT: the first n tokens.  RECENT: the last n
+    tokens.  CALLER: rows drawn outside (the ablation's random sampling), n distinct indices given in
+    `caller_rows`, used in the order given.  The last three are the alternatives the paper's
+    query-subset ablation compares the uniform rule with."""
     n = min(n_obs, n_k)
-    return np.array([(m * n_k) // n for m in range(n)], dtype=np.int64)
+    if sampler == UNIFORM:
+        return np.array([(m * n_k) // n for m in range(n)], dtype=np.int64)
+    if sampler == INIT:
+        return np.arange(n, dtype=np.int64)
+    if sampler == RECENT:
+        return np.arange(n_k - n, n_k, dtype=np.int64)
+    if sampler == CALLER:
+        rows = np.asarray(caller_rows, dtype=np.int64)
+        if rows.shape != (n,) or rows.min() < 0 or rows.max() >= n_k or len(set(rows.tolist())) != n:
+            raise ValueError("caller_rows must hold min(N_obs, N_k) distinct rows of the current scale")
+        return rows
+    raise ValueError(sampler)
 
 
 def softmax_rows(z: np.ndarray) -> np.ndarray:
@@ -138,7 +158,8 @@ class HackOracle:
     def __init__(self, n_layers: int, n_heads: int, batch: int, head_dim: int,
                  sides: Sequence[int], head_is_contextual: np.ndarray,
                  budget_c: int, budget_s: int, n_obs: int = 32, n_init_scales: int = 2,
-                 sm_scale: Optional[float] = None, overflow_policy: int = KEEP_PROTECTED):
+                 sm_scale: Optional[float] = None, overflow_policy: int = KEEP_PROTECTED,
+                 obs_sampler: int = UNIFORM, obs_rows: Optional[Sequence[Sequence[int]]] = None):
         self.L, self.H, self.b, self.D = n_layers, n_heads, batch, head_dim
         self.sides = tuple(int(s) for s in sides)
         self.N = tuple(s * s for s in self.sides)
@@ -148,6 +169,8 @@ class HackOracle:
         self.n_obs, self.n_init_scales = int(n_obs), int(n_init_scales)
         self.sm_scale = float(sm_scale) if sm_scale else 1.0 / math.sqrt(head_dim)
         self.policy = overflow_policy
+        self.obs_sampler = obs_sampler
+        self.obs_rows = obs_rows            # CALLER: one row list per scale
         self.counters = Counters()
         self.reset()
 
@@ -192,7 +215,8 @@ class HackOracle:
             compressed = False
         else:
             compressed = True
-            obs = observation_rows(n_k, self.n_obs)
+            obs = observation_rows(n_k, self.n_obs, self.obs_sampler,
+                                   self.obs_rows[scale] if self.obs_sampler == CALLER else None)
             scores = subset_attention_scores(q[obs], k_c, self.sm_scale)
             self.counters.score_pairs += obs.shape[0] * t_cand
             s_sel = scores if scores_override is None else np.asarray(scores_override, dtype=np.float64)

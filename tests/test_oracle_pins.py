@@ -99,6 +99,55 @@ def test_observation_rows_uniform_and_complete():
     assert r[-1] < 100
 
 
+def test_observation_rows_of_the_ablation_samplers():
+    """Query-subset ablation: first n, last n, caller-drawn rows; every rule degenerates to all
+    rows when the scale has no more than N_obs tokens."""
+    assert list(ho.observation_rows(10, 4, ho.UNIFORM)) == [0, 2, 5, 7]
+    assert list(ho.observation_rows(10, 4, ho.INIT)) == [0, 1, 2, 3]
+    assert list(ho.observation_rows(10, 4, ho.RECENT)) == [6, 7, 8, 9]
+    assert list(ho.observation_rows(10, 4, ho.CALLER, [9, 0, 4, 3])) == [9, 0, 4, 3]
+    for sampler in (ho.UNIFORM, ho.INIT, ho.RECENT):
+        assert list(ho.observation_rows(9, 32, sampler)) == list(range(9))
+    for bad in ([0, 1, 2], [0, 1, 2, 2], [0, 1, 2, 10], [-1, 1, 2, 3]):
+        with pytest.raises(ValueError):
+            ho.observation_rows(10, 4, ho.CALLER, bad)
+
+
+def test_sampler_decides_which_key_a_contextual_head_keeps():
+    """Two planted keys: the first half of the queries looks at key 0, the second half at key 1.
+    With one slot for old entries, the first-n rule keeps key 0, the last-n rule key 1, and caller
+    rows taken from one half or the other reproduce the two; computed against a direct column sum."""
+    D, n_k = 8, 16
+    rng = np.random.default_rng(5)
+    e0, e1 = np.eye(D)[0] * 6.0, np.eye(D)[1] * 6.0
+    k_new = rng.normal(size=(n_k, D)) * 0.05
+    k_new[0], k_new[1] = e0, e1
+    q = rng.normal(size=(n_k, D)) * 0.05
+    q[: n_k // 2] += e0
+    q[n_k // 2:] += e1
+    v = rng.normal(size=(n_k, D))
+    for sampler, rows, expect in ((ho.INIT, None, 0), (ho.RECENT, None, 1),
+                                  (ho.CALLER, [[3, 1, 6, 0]], 0), (ho.CALLER, [[15, 9, 12, 10]], 1)):
+        orc = ho.HackOracle(1, 1, 1, D, (4,), np.array([[1]]), budget_c=1, budget_s=1, n_obs=4,
+                            obs_sampler=sampler, obs_rows=rows)
+        _, res = orc.head_step(0, 0, 0, 0, q, k_new, v)
+        used = ho.observation_rows(n_k, 4, sampler, rows[0] if rows else None)
+        z = (q[used] @ k_new.T) / math.sqrt(D)
+        a = np.exp(z - z.max(axis=1, keepdims=True))
+        a /= a.sum(axis=1, keepdims=True)
+        assert int(np.argmax(a.sum(axis=0))) == expect
+        assert list(res.keep) == [expect]
+
+
+def test_caller_rows_order_does_not_change_scores():
+    rng = np.random.default_rng(6)
+    q, k = rng.normal(size=(40, 16)), rng.normal(size=(70, 16))
+    rows = [31, 2, 17, 8, 25]
+    s1 = ho.subset_attention_scores(q[ho.observation_rows(40, 5, ho.CALLER, rows)], k, 0.25)
+    s2 = ho.subset_attention_scores(q[ho.observation_rows(40, 5, ho.CALLER, sorted(rows))], k, 0.25)
+    np.testing.assert_allclose(s1, s2, rtol=1e-13)
+
+
 # ------------------------------------------------------------------ P3: brute-force selection
 def _best_subset_exhaustive(s, n):
     """argmax-n subset by exhaustive enumeration; among equal sums the lexicographically

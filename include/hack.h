@@ -62,6 +62,14 @@ typedef enum { HACK_F32 = 0, HACK_BF16 = 1 } hack_dtype_t;
 enum { HACK_OVERFLOW_KEEP_PROTECTED = 0, /* keep every protected entry, exceed B_S */
        HACK_OVERFLOW_COMPETE = 1 };      /* protect only the initial scales; keep exactly B_S */
 
+/* Which n = min(N_obs, N_k) queries of the current scale form the subset Q~ of Eq. 9.  The method
+ * uses uniform spacing; the others are the alternatives of the paper's query-subset ablation. */
+enum { HACK_OBS_UNIFORM = 0, /* floor(m * N_k / n), m = 0..n-1 */
+       HACK_OBS_INIT = 1,    /* the first n tokens of the scale */
+       HACK_OBS_RECENT = 2,  /* the last n tokens of the scale */
+       HACK_OBS_CALLER = 3 };/* rows given per scale with hack_set_obs_rows (random sampling: the
+                                caller draws them) */
+
 typedef struct {
   int32_t n_layers, n_heads, head_dim, batch; /* head_dim in {64, 128} */
   int32_t n_scales;
@@ -75,6 +83,7 @@ typedef struct {
   float sm_scale;                    /* softmax scale; 0 selects 1/sqrt(head_dim) */
   int32_t overflow_policy;           /* HACK_OVERFLOW_* */
   int32_t device;                    /* CUDA device ordinal */
+  int32_t obs_sampler;               /* HACK_OBS_*; 0 = the method's uniform rule */
 } hack_config_t;
 
 /* Host-side plan of one step of one layer (all lengths in entries per head). */
@@ -108,6 +117,14 @@ HACK_API hack_status_t hack_split_budget(int32_t budget, double alpha, int32_t r
 HACK_API hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out);
 /* Release everything; synchronises the device first.  NULL is accepted. */
 HACK_API hack_status_t hack_free_cache(hack_cache_t* cache);
+/* HACK_OBS_CALLER only: the query rows that form Q~ (Eq. 9) at `scale`, for every layer, batch
+ * element and head.  rows: host, n = min(N_obs, N_k) distinct indices in [0, N_k), used in the
+ * order given (the scores do not depend on the order).  Copied to the device synchronously: a
+ * set-up call, made before the steps of that scale are enqueued; the rows stay in force across
+ * hack_reset.  A step that has to score while its scale has no rows fails with HACK_ERR_STATE.
+ * INVALID_ARG for a wrong n, an index out of range or a repeated index; STATE if the cache was
+ * not created with HACK_OBS_CALLER. */
+HACK_API hack_status_t hack_set_obs_rows(hack_cache_t* cache, int32_t scale, const int32_t* rows, int32_t n);
 /* New image: all layers back to scale 0 with empty caches.  Enqueues nothing. */
 HACK_API hack_status_t hack_reset(hack_cache_t* cache);
 

@@ -16,10 +16,11 @@ HACK_OK, HACK_ERR_INVALID_ARG, HACK_ERR_UNSUPPORTED, HACK_ERR_OOM, HACK_ERR_CUDA
     HACK_ERR_TIMEOUT = range(7)
 HACK_F32, HACK_BF16 = 0, 1
 HACK_OVERFLOW_KEEP_PROTECTED, HACK_OVERFLOW_COMPETE = 0, 1
+HACK_OBS_UNIFORM, HACK_OBS_INIT, HACK_OBS_RECENT, HACK_OBS_CALLER = 0, 1, 2, 3
 RULE_FRACTION, RULE_RATIO = 0, 1
 
 EXPORTS = (
-    "hack_split_budget", "hack_init_cache", "hack_free_cache", "hack_reset", "hack_get_limits",
+    "hack_split_budget", "hack_init_cache", "hack_free_cache", "hack_reset", "hack_set_obs_rows", "hack_get_limits",
     "hack_step_info", "hack_score", "hack_select", "hack_compact", "hack_attend", "hack_scale_step",
     "hack_scale_step_host", "hack_score_noalloc", "hack_get_lengths", "hack_read_head", "hack_kv_bytes",
     "hack_launch_count", "hack_stage_timing", "hack_stage_times", "hack_poll_status", "hack_last_error",
@@ -32,7 +33,7 @@ class HackConfig(C.Structure):
         ("n_scales", C.c_int32), ("scale_sides", C.POINTER(C.c_int32)), ("dtype", C.c_int32),
         ("head_is_contextual", C.POINTER(C.c_uint8)), ("budget_c", C.c_int32), ("budget_s", C.c_int32),
         ("n_obs", C.c_int32), ("n_init_scales", C.c_int32), ("sm_scale", C.c_float),
-        ("overflow_policy", C.c_int32), ("device", C.c_int32),
+        ("overflow_policy", C.c_int32), ("device", C.c_int32), ("obs_sampler", C.c_int32),
     ]
 
 
@@ -66,6 +67,7 @@ def _load() -> C.CDLL:
         "hack_init_cache": [C.POINTER(HackConfig), C.POINTER(vp)],
         "hack_free_cache": [vp],
         "hack_reset": [vp],
+        "hack_set_obs_rows": [vp, i32, C.POINTER(i32), i32],
         "hack_get_limits": [vp, C.POINTER(HackLimits)],
         "hack_step_info": [vp, i32, i32, C.POINTER(HackStepInfo)],
         "hack_score": [vp, i32, i32, vp, vp, vp, vp],
@@ -130,7 +132,8 @@ class HackCache:
     def __init__(self, n_layers: int, n_heads: int, head_dim: int, batch: int, sides: Sequence[int],
                  dtype: int, head_is_contextual, budget_c: int, budget_s: int, n_obs: int = 32,
                  n_init_scales: int = 2, sm_scale: float = 0.0,
-                 overflow_policy: int = HACK_OVERFLOW_KEEP_PROTECTED, device: int = 0):
+                 overflow_policy: int = HACK_OVERFLOW_KEEP_PROTECTED, device: int = 0,
+                 obs_sampler: int = HACK_OBS_UNIFORM):
         self._h = C.c_void_p()
         sides_arr = (C.c_int32 * len(sides))(*[int(s) for s in sides])
         flat = [int(v) for v in (head_is_contextual.reshape(-1).tolist()
@@ -139,7 +142,8 @@ class HackCache:
         if len(flat) != n_layers * n_heads:
             raise ValueError("head_is_contextual must have n_layers*n_heads entries")
         cfg = HackConfig(n_layers, n_heads, head_dim, batch, len(sides), sides_arr, dtype, mask_arr,
-                         budget_c, budget_s, n_obs, n_init_scales, sm_scale, overflow_policy, device)
+                         budget_c, budget_s, n_obs, n_init_scales, sm_scale, overflow_policy, device,
+                         obs_sampler)
         _check(lib.hack_init_cache(C.byref(cfg), C.byref(self._h)))
         self.n_layers, self.n_heads, self.head_dim, self.batch = n_layers, n_heads, head_dim, batch
         self.dtype = dtype
@@ -158,6 +162,10 @@ class HackCache:
             self.close()
         except Exception:
             pass
+
+    def hack_set_obs_rows(self, scale: int, rows: Sequence[int]) -> None:
+        arr = (C.c_int32 * len(rows))(*[int(r) for r in rows])
+        _check(lib.hack_set_obs_rows(self._h, scale, arr, len(rows)))
 
     def hack_reset(self) -> None:
         _check(lib.hack_reset(self._h))

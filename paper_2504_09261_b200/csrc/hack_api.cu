@@ -72,6 +72,8 @@ struct hack_cache {
   hack::Scratch scratch{};
   int* status = nullptr;
   int32_t* n_old = nullptr;                     // [b*H] scratch of the compaction kernels
+  int32_t* obs_rows = nullptr;                  // HACK_OBS_CALLER: [n_scales][kMaxObs] query rows of Q~
+  std::vector<uint8_t> obs_rows_set;            // per scale: rows were supplied
   std::vector<TensorMapBox> k_maps, v_maps;     // per layer, bf16 caches only
   int32_t* head_order = nullptr;                // [L][2][b*H]: [0] structural heads first, [1] contextual first
   // host-buffer entry point: kHostSlots staging sets (q, k, v, o) cycled call by call, copies on
@@ -150,6 +152,10 @@ hack::StepArgs make_args(const hack_cache* c, int layer, int scale, const hack_s
   a.kept[0] = p.kept_s;     a.kept[1] = p.kept_c;
   a.trig[0] = p.triggered_s; a.trig[1] = p.triggered_c;
   a.n_obs_rows = p.n_obs_rows;
+  // the query subset of Eq. 9: uniform spacing, or one of the ablation's alternatives
+  a.obs_first = c->cfg.obs_sampler == HACK_OBS_RECENT ? p.n_new - p.n_obs_rows : 0;
+  a.obs_span = c->cfg.obs_sampler == HACK_OBS_UNIFORM ? p.n_new : p.n_obs_rows;
+  a.obs_rows = c->cfg.obs_sampler == HACK_OBS_CALLER ? c->obs_rows + (size_t)scale * hack::kMaxObs : nullptr;
   a.sm_scale = c->sm_scale;
   a.t_init = c->t_init;
   a.protect_new = (c->cfg.overflow_policy == HACK_OVERFLOW_KEEP_PROTECTED) || scale < c->cfg.n_init_scales;
@@ -269,6 +275,7 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return fail(HACK_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
   if (cfg->dtype != HACK_F32 && cfg->dtype != HACK_BF16) return fail(HACK_ERR_UNSUPPORTED, "dtype must be HACK_F32 or HACK_BF16");
   if (cfg->n_obs < 1 || cfg->n_obs > hack::kMaxObs) return fail(HACK_ERR_UNSUPPORTED, "n_obs must be in 1..32");
+  if (cfg->obs_sampler < HACK_OBS_UNIFORM || cfg->obs_sampler > HACK_OBS_CALLER) return fail(HACK_ERR_INVALID_ARG, "unknown obs_sampler");
   for (int k = 0; k < cfg->n_scales; ++k)
     if (cfg->scale_sides[k] < 1 || cfg->scale_sides[k] > 1024) return fail(HACK_ERR_INVALID_ARG, "scale side out of range (1..1024)");
   for (int i = 0; i < cfg->n_layers * cfg->n_heads; ++i)
@@ -391,6 +398,11 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
     HACK_TRY(cudaMemcpy(c->head_order, order.data(), order.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
   }
   HACK_TRY(cudaMalloc(&c->n_old, (size_t)bh * sizeof(int32_t)));
+  if (cfg->obs_sampler == HACK_OBS_CALLER) {
+    HACK_TRY(cudaMalloc(&c->obs_rows, (size_t)cfg->n_scales * hack::kMaxObs * sizeof(int32_t)));
+    HACK_TRY(cudaMemset(c->obs_rows, 0, (size_t)cfg->n_scales * hack::kMaxObs * sizeof(int32_t)));
+    c->obs_rows_set.assign(cfg->n_scales, 0);
+  }
   HACK_TRY(cudaMalloc(&c->status, sizeof(int)));
   HACK_TRY(cudaMemset(c->status, 0, sizeof(int)));
   HACK_TRY(cudaDeviceSynchronize());
@@ -408,6 +420,7 @@ hack_status_t hack_free_cache(hack_cache_t* c) {
   cudaFree(c->scratch.logits); cudaFree(c->scratch.partials); cudaFree(c->status);
   cudaFree(c->head_order);
   cudaFree(c->n_old);
+  cudaFree(c->obs_rows);
   for (int sl = 0; sl < hack_cache::kHostSlots; ++sl) {
     for (int i = 0; i < 4; ++i) cudaFree(c->stage[sl][i]);
     if (c->ev_in[sl]) cudaEventDestroy(c->ev_in[sl]);
@@ -418,6 +431,23 @@ hack_status_t hack_free_cache(hack_cache_t* c) {
   if (c->d2h_stream) cudaStreamDestroy(c->d2h_stream);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   delete c;
+  return HACK_OK;
+}
+
+hack_status_t hack_set_obs_rows(hack_cache_t* c, int32_t scale, const int32_t* rows, int32_t n) {
+  if (!c || !rows) return fail(HACK_ERR_INVALID_ARG, "cache or rows is NULL");
+  if (c->cfg.obs_sampler != HACK_OBS_CALLER) return fail(HACK_ERR_STATE, "the cache was not created with HACK_OBS_CALLER");
+  if (scale < 0 || scale >= c->cfg.n_scales) return fail(HACK_ERR_INVALID_ARG, "scale out of range");
+  const int n_new = c->n_tok[scale];
+  if (n != std::min(c->cfg.n_obs, n_new)) return fail(HACK_ERR_INVALID_ARG, "n must be min(N_obs, N_k)");
+  for (int i = 0; i < n; ++i) {
+    if (rows[i] < 0 || rows[i] >= n_new) return fail(HACK_ERR_INVALID_ARG, "observation row out of range");
+    for (int j = 0; j < i; ++j)
+      if (rows[j] == rows[i]) return fail(HACK_ERR_INVALID_ARG, "observation rows must be distinct");
+  }
+  HACK_CUDA(cudaSetDevice(c->cfg.device));
+  HACK_CUDA(cudaMemcpy(c->obs_rows + (size_t)scale * hack::kMaxObs, rows, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice));
+  c->obs_rows_set[scale] = 1;
   return HACK_OK;
 }
 
@@ -453,6 +483,8 @@ hack_status_t hack_score(hack_cache_t* c, int32_t layer, int32_t scale, const vo
   if (misaligned(q) || misaligned(k_new) || misaligned(scores)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
   hack_step_info_t p;
   plan_step(c, c->layers[layer], scale, &p);
+  if (c->cfg.obs_sampler == HACK_OBS_CALLER && (p.triggered_c || p.triggered_s) && !c->obs_rows_set[scale])
+    return fail(HACK_ERR_STATE, "HACK_OBS_CALLER: no observation rows were set for this scale (hack_set_obs_rows)");
   const hack::StepArgs a = make_args(c, layer, scale, p);
   StageScope ts(c, (cudaStream_t)stream, 0);
   const int n = hack::launch_score(a, c->cfg.dtype, q, k_new, scores, c->scratch, (cudaStream_t)stream);
@@ -532,6 +564,8 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
   cudaStream_t st = (cudaStream_t)stream;
   hack_step_info_t p;
   plan_step(c, c->layers[layer], scale, &p);
+  if (c->cfg.obs_sampler == HACK_OBS_CALLER && (p.triggered_c || p.triggered_s) && !c->obs_rows_set[scale])
+    return fail(HACK_ERR_STATE, "HACK_OBS_CALLER: no observation rows were set for this scale (hack_set_obs_rows)");
   const hack::StepArgs a = make_args(c, layer, scale, p);
   const bool any = p.triggered_c || p.triggered_s;
   int n = 0, r;

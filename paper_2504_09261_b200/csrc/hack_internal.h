@@ -25,6 +25,8 @@ struct StepArgs {
   int kept[2];          // length after the step
   int trig[2];          // compression triggered for this type
   int n_obs_rows;       // min(N_obs, N_k)
+  int obs_first, obs_span;      // observation row i = obs_first + floor(i * obs_span / n_obs_rows) ...
+  const int32_t* obs_rows;      // ... unless the caller supplied the rows (device, [n_obs_rows])
   float sm_scale;
   int t_init;           // tokens in the always-kept leading scales (structural heads)
   int protect_new;      // structural heads: the new scale's tokens are protected
@@ -97,6 +99,10 @@ inline void launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
   cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 #if defined(__CUDACC__)
+// Query row that serves as observation row i (Eq. 9's subset Q~).
+__device__ __forceinline__ int obs_row(const StepArgs& a, int i) {
+  return a.obs_rows ? a.obs_rows[i] : a.obs_first + (int)(((long long)i * a.obs_span) / a.n_obs_rows);
+}
 __device__ __forceinline__ void pdl_wait() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");

@@ -60,12 +60,12 @@ score_logits_kernel(const StepArgs a, const T* __restrict__ q, const T* __restri
   float* zt = reinterpret_cast<float*>(ks);                             // reused: [32][128]
 
   const T* kp = static_cast<const T*>(a.k_plane);
-  // observation rows: floor(m * N_k / n)
+  // observation rows: floor(m * N_k / n) under the uniform rule
   for (int v = tid; v < kMaxObs * ROWV; v += kScoreChunk) {
     const int i = v / ROWV, c = v % ROWV;
     float f[VEC];
     if (i < a.n_obs_rows) {
-      const int row = (int)(((long long)i * a.n_new) / a.n_obs_rows);
+      const int row = obs_row(a, i);
       const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)bh * a.n_new + row) * D + c * VEC);
       Elem<T>::unpack(raw, f);
     } else {

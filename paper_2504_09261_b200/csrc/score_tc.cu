@@ -111,12 +111,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_const
     fence_barrier_init();
     fence_proxy_async();
   }
-  // observation rows floor(i * N_k / n) into the swizzled B tile; unused rows are zero
+  // observation rows (floor(i * N_k / n) under the uniform rule) into the swizzled B tile; unused rows are zero
   for (int v = tid; v < kMaxObs * (D / 8); v += kScoreThreads) {
     const int i = v / (D / 8), c = v % (D / 8);
     uint4 val = make_uint4(0, 0, 0, 0);
     if (i < a.n_obs_rows) {
-      const int row = (int)(((long long)i * a.n_new) / a.n_obs_rows);
+      const int row = obs_row(a, i);
       val = *reinterpret_cast<const uint4*>(q + ((size_t)bh * a.n_new + row) * D + c * 8);
     }
     const uint32_t off = (c / 8) * Q_SUB_BYTES + i * 128 + (((c % 8) ^ (i & 7)) << 4);

@@ -51,14 +51,18 @@ def _torch_dtype(cfg: WorkloadConfig):
 
 
 def make_cache(cfg: WorkloadConfig, mask: np.ndarray, policy: int = 0, budget_c: Optional[int] = None,
-               budget_s: Optional[int] = None, device: int = 0):
+               budget_s: Optional[int] = None, device: int = 0, obs_sampler: int = 0, obs_rows=None):
     from paper_2504_09261_b200 import HACK_BF16, HACK_F32, HackCache
-    return HackCache(cfg.n_layers, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides,
-                     HACK_F32 if cfg.dtype == "f32" else HACK_BF16, mask,
-                     cfg.budget_c if budget_c is None else budget_c,
-                     cfg.budget_s if budget_s is None else budget_s,
-                     n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, overflow_policy=policy,
-                     device=device)
+    cache = HackCache(cfg.n_layers, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides,
+                      HACK_F32 if cfg.dtype == "f32" else HACK_BF16, mask,
+                      cfg.budget_c if budget_c is None else budget_c,
+                      cfg.budget_s if budget_s is None else budget_s,
+                      n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, overflow_policy=policy,
+                      device=device, obs_sampler=obs_sampler)
+    if obs_rows is not None:
+        for k, rows in enumerate(obs_rows):
+            cache.hack_set_obs_rows(k, rows)
+    return cache
 
 
 def sample_heads(cfg: WorkloadConfig, layer: int, n: Optional[int]) -> List[Tuple[int, int]]:
@@ -78,7 +82,8 @@ def _rows_bytes(arr64: np.ndarray, tdt) -> bytes:
 def run_parity(cfg: WorkloadConfig, layers: Sequence[int], fused: bool = False,
                heads_per_layer: Optional[int] = None, policy: int = 0,
                budget_c: Optional[int] = None, budget_s: Optional[int] = None,
-               scales: Optional[int] = None, check_rows: bool = True) -> ParityReport:
+               scales: Optional[int] = None, check_rows: bool = True,
+               obs_sampler: int = 0, obs_rows=None) -> ParityReport:
     dev = torch.device("cuda:0")
     tdt = _torch_dtype(cfg)
     gen = SyntheticQKV(cfg)
@@ -86,9 +91,10 @@ def run_parity(cfg: WorkloadConfig, layers: Sequence[int], fused: bool = False,
     b_c = cfg.budget_c if budget_c is None else budget_c
     b_s = cfg.budget_s if budget_s is None else budget_s
     orc = ho.HackOracle(cfg.n_layers, cfg.n_heads, cfg.batch, cfg.head_dim, cfg.sides, mask, b_c, b_s,
-                        n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, overflow_policy=policy)
-    staged = make_cache(cfg, mask, policy, b_c, b_s)
-    twin = make_cache(cfg, mask, policy, b_c, b_s) if fused else None
+                        n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, overflow_policy=policy,
+                        obs_sampler=obs_sampler, obs_rows=obs_rows)
+    staged = make_cache(cfg, mask, policy, b_c, b_s, obs_sampler=obs_sampler, obs_rows=obs_rows)
+    twin = make_cache(cfg, mask, policy, b_c, b_s, obs_sampler=obs_sampler, obs_rows=obs_rows) if fused else None
     rep = ParityReport(cfg.name)
     bh = cfg.batch * cfg.n_heads
     H = cfg.n_heads

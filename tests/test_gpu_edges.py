@@ -68,6 +68,58 @@ def test_single_observation_row_and_single_scale():
     _ok(rep)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("sampler", ["init", "recent", "caller"])
+def test_query_subset_rules_of_the_ablation(sampler, dtype):
+    """The alternatives the paper's query-subset ablation compares with uniform spacing (first n,
+    last n, random rows drawn by the caller) against the oracle under the same rule, with N_obs = 8
+    and 32 so that both subset sizes of the size ablation's range and a ragged last scale occur."""
+    import paper_2504_09261_b200 as hb
+    from workloads import random_observation_rows
+    from tests.parity_util import run_parity
+    code = {"init": hb.HACK_OBS_INIT, "recent": hb.HACK_OBS_RECENT, "caller": hb.HACK_OBS_CALLER}[sampler]
+    for n_obs in (8, 32):
+        cfg = _custom(1 if dtype == "bf16" else 0, n_obs=n_obs, n_heads=4, batch=1, dtype=dtype,
+                      sides=(1, 2, 3, 5, 8, 13, 19))
+        rows = random_observation_rows(cfg, seed=n_obs) if sampler == "caller" else None
+        rep = run_parity(cfg, layers=[0], fused=True, budget_c=60, budget_s=260, obs_sampler=code, obs_rows=rows)
+        _ok(rep)
+        assert rep.compressed_heads > 0
+
+
+def test_caller_rows_are_checked_and_required():
+    import paper_2504_09261_b200 as hb
+    import torch
+    from workloads import SyntheticQKV
+    cfg = _custom(0, n_heads=2, batch=1, sides=(1, 2, 6), n_obs=4)
+    gen = SyntheticQKV(cfg)
+    mask = gen.head_is_contextual.numpy()
+    uniform = hb.HackCache(1, 2, cfg.head_dim, 1, cfg.sides, hb.HACK_F32, mask, 4, 8, n_obs=4)
+    with pytest.raises(hb.HackError) as e:
+        uniform.hack_set_obs_rows(2, [0, 1, 2, 3])
+    assert e.value.status == 5
+    uniform.close()
+    cache = hb.HackCache(1, 2, cfg.head_dim, 1, cfg.sides, hb.HACK_F32, mask, 4, 8, n_obs=4,
+                         obs_sampler=hb.HACK_OBS_CALLER)
+    for bad in ([0, 1, 2], [0, 1, 2, 2], [0, 1, 2, 36], [-1, 1, 2, 3]):
+        with pytest.raises(hb.HackError) as e:
+            cache.hack_set_obs_rows(2, bad)
+        assert e.value.status == 1
+    dev = torch.device("cuda:0")
+    for k in range(3):
+        q, kk, v = (t.to(dev) for t in gen.qkv(0, k))
+        out = torch.empty_like(q)
+        if cache.hack_step_info(0, k).triggered_c:
+            with pytest.raises(hb.HackError) as e:           # scoring without rows for this scale
+                cache.hack_scale_step(0, k, q, kk, v, out)
+            assert e.value.status == 5
+            cache.hack_set_obs_rows(k, [35, 0, 7, 20] if k == 2 else list(range(min(4, cfg.sides[k] ** 2))))
+        cache.hack_scale_step(0, k, q, kk, v, out)
+    torch.cuda.synchronize()
+    assert cache.hack_get_lengths(0) == [4, 41]      # structural head: 5 initial + 36 new tokens are protected
+    cache.close()
+
+
 def test_graph_replay_reproduces_direct_calls():
     """bench.py times CUDA-graph replays of the hack_scale_step calls; a replay has to write the
     same bytes as the direct calls did (the length plan is fixed, so a captured loop is complete)."""

@@ -5,4 +5,4 @@ Q/K/V tensors).  It holds none of the method's arithmetic: no scoring, selection
 attention or budget splitting lives here.
 """
 from .configs import WorkloadConfig, get_config, SCHEDULES, list_configs  # noqa: F401
-from .synthetic import SyntheticQKV  # noqa: F401
+from .synthetic import SyntheticQKV, random_observation_rows  # noqa: F401

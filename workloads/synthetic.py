@@ -202,3 +202,17 @@ class SyntheticQKV:
 
 # Layer count of the named workloads (the global head permutation is drawn over the full stack).
 _FULL_LAYERS = {0: 1, 1: 16, 2: 30, 3: 32, 4: 40}
+
+
+def random_observation_rows(cfg: WorkloadConfig, seed: int = 0) -> list:
+    """Per scale, min(N_obs, N_k) distinct query rows drawn without replacement (the random-sampling
+    arm of the query-subset ablation).  The draw is an input of the method, so it is made here, once,
+    and handed to both the CPU oracle and the GPU library."""
+    import numpy as np
+    rng = np.random.default_rng(cfg.seed * 1000003 + seed)
+    rows = []
+    for side in cfg.sides:
+        n_k = side * side
+        n = min(cfg.n_obs, n_k)
+        rows.append([int(r) for r in rng.choice(n_k, size=n, replace=False)])
+    return rows

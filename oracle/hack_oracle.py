@@ -13,6 +13,8 @@ the tests, the smoke check and the CPU-baseline leg of the benchmark may use it.
 Parity pins (see tests/test_oracle_*.py): full-budget == vanilla attention (Eq. 3-4), softmax
 row sums, brute-force subset selection, protected-scale invariants, the closed forms of the
 complexity analysis (Eq. 12-22), convexity and permutation invariance of the attention output.
+Offline head classification (Eq. 6) is here too: attention_variance and classify_heads, pinned by
+closed forms (identity and uniform attention) and by recovering a planted head mask.
 Parity unpinned (the paper is silent; only self-consistency is tested): the overflow rule when
 B_S < N_init + N_k, the exact stride of the "uniform" query sample, the budget rounding rule.
 """
@@ -263,6 +265,29 @@ class HackOracle:
         self.next_scale[layer] = scale + 1
         self.counters.peak_entries = max(self.counters.peak_entries, self._live)
         return out, records
+
+
+# --------------------------------------------------------------------------- offline head classification
+def attention_variance(q: np.ndarray, k: np.ndarray, sm_scale: float) -> float:
+    """sigma = sum_j Var_i A[i, j] for one head (Eq. 6): A = Softmax(sm_scale * Q K^T) is the
+    attention matrix of the step's queries (rows) over the cached keys (columns); the variance of a
+    column is taken over the queries, as the population variance (mean of squares minus squared
+    mean; the paper does not say which normalisation, and the ranking does not depend on it)."""
+    a = softmax_rows(sm_scale * (q @ k.T))
+    return float(np.var(a, axis=0).sum())
+
+
+def classify_heads(sigma: np.ndarray, alpha: float) -> np.ndarray:
+    """Head types from the variance matrix sigma [L, H] (averaged over samples by the caller): all
+    heads are ranked globally by sigma and the round(alpha * L * H) lowest become contextual (1),
+    the others structural (0).  Equal values are ranked by (layer, head)."""
+    sigma = np.asarray(sigma, dtype=np.float64)
+    flat = sigma.reshape(-1)
+    n_ctx = int(math.floor(alpha * flat.shape[0] + 0.5))
+    order = np.argsort(flat, kind="stable")
+    mask = np.zeros(flat.shape[0], dtype=np.uint8)
+    mask[order[:n_ctx]] = 1
+    return mask.reshape(sigma.shape)
 
 
 # --------------------------------------------------------------------------- vanilla reference

@@ -389,3 +389,61 @@ def test_mean_kept_length_within_budget():
         assert orc.stored_lengths(0).mean() <= B
     assert orc.counters.overflows == 0
     assert orc.counters.peak_entries == orc.stored_lengths(0).sum()
+
+
+# ------------------------------------------------------------------ Eq. 6: attention variance
+def test_attention_variance_closed_forms():
+    """Uniform attention has no column variance; attention that is (nearly) a permutation matrix has
+    sigma = T * (1/N)(1 - 1/N) = 1 - 1/N for N = T; identical query rows give zero whatever the keys."""
+    n, d = 12, 12
+    k = np.eye(d) * 200.0                      # query i = key i: softmax row i is one-hot to 1e-80
+    assert ho.attention_variance(np.eye(d), k, 1.0) == pytest.approx(1.0 - 1.0 / n, rel=1e-12)
+    assert ho.attention_variance(np.zeros((n, d)), k, 1.0) == pytest.approx(0.0, abs=1e-30)
+    rng = np.random.default_rng(3)
+    q1 = np.repeat(rng.normal(size=(1, d)), n, axis=0)
+    assert ho.attention_variance(q1, rng.normal(size=(30, d)), 0.3) == pytest.approx(0.0, abs=1e-30)
+
+
+def test_attention_variance_matches_loops():
+    rng = np.random.default_rng(4)
+    q, k = rng.normal(size=(7, 5)), rng.normal(size=(9, 5))
+    a = np.zeros((7, 9))
+    for i in range(7):
+        z = [0.4 * sum(q[i, t] * k[j, t] for t in range(5)) for j in range(9)]
+        den = sum(math.exp(x) for x in z)
+        for j in range(9):
+            a[i, j] = math.exp(z[j]) / den
+    sigma = 0.0
+    for j in range(9):
+        mean = sum(a[i, j] for i in range(7)) / 7
+        sigma += sum((a[i, j] - mean) ** 2 for i in range(7)) / 7
+    assert ho.attention_variance(q, k, 0.4) == pytest.approx(sigma, rel=1e-12)
+    # transposing the roles of rows and columns is a different number (variance over queries, not keys)
+    assert abs(float(np.var(a, axis=1).sum()) - sigma) > 1e-3
+
+
+def test_classify_heads_ranks_globally():
+    sigma = np.array([[0.9, 0.1, 0.5], [0.2, 0.8, 0.1]])
+    assert ho.classify_heads(sigma, 0.5).tolist() == [[0, 1, 0], [1, 0, 1]]
+    assert ho.classify_heads(sigma, 1 / 3).tolist() == [[0, 1, 0], [0, 0, 1]]     # per-layer ratio varies
+    assert ho.classify_heads(np.zeros((2, 2)), 0.5).tolist() == [[1, 1], [0, 0]]   # ties: (layer, head) order
+
+
+def test_variance_ranking_recovers_the_planted_head_types():
+    """The synthetic workloads plant vertical patterns in contextual heads and position-following
+    ones in structural heads; Eq. 6 on the last scale's full attention matrix must separate them."""
+    from workloads import SyntheticQKV, get_config
+    cfg = get_config(0, n_layers=2)
+    gen = SyntheticQKV(cfg)
+    mask = gen.head_is_contextual.numpy().astype(np.uint8)
+    sigma = np.zeros((cfg.n_layers, cfg.n_heads))
+    last = cfg.n_scales - 1
+    for l in range(cfg.n_layers):
+        ks = [gen.qkv(l, s)[1].double().numpy() for s in range(cfg.n_scales)]
+        q = gen.qkv(l, last)[0].double().numpy()
+        for h in range(cfg.n_heads):
+            k_all = np.concatenate([x[0, h] for x in ks], axis=0)
+            sigma[l, h] = ho.attention_variance(q[0, h], k_all, 1.0 / math.sqrt(cfg.head_dim))
+    alpha = float(mask.mean())
+    assert ho.classify_heads(sigma, alpha).tolist() == mask.tolist()
+    assert sigma[mask == 1].max() < sigma[mask == 0].min()

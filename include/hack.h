@@ -163,6 +163,25 @@ HACK_API hack_status_t hack_compact(hack_cache_t* cache, int32_t layer, int32_t 
 HACK_API hack_status_t hack_attend(hack_cache_t* cache, int32_t layer, int32_t scale, const void* q,
                           void* out, void* stream);
 
+/* hack_attend that also returns the attention variance of every head (Eq. 6, offline head
+ * classification): sigma[b*H + h] = sum_j Var_i A[i, j], A = Softmax(sm_scale * Q K^T) the attention
+ * matrix of this step's queries (rows) over the head's cache as it stands (columns), Var the
+ * population variance over the queries.  For Eq. 6 proper, create the cache with budgets >= T_K, so
+ * that nothing is evicted, and call this at the last scale: A is then the N_K x T_K matrix of the
+ * final generation step.  sigma: device, [batch*n_heads] floats, written on `stream`.  State rules
+ * of hack_attend.  UNSUPPORTED unless the cache is bf16 and the scale has at least 32 tokens (and
+ * batch*n_heads*N_k >= 128): the statistics come from the tensor-core attention kernel. */
+HACK_API hack_status_t hack_attend_variance(hack_cache_t* cache, int32_t layer, int32_t scale, const void* q,
+                                   void* out, float* sigma, void* stream);
+
+/* Head types from the variance matrix (Eq. 6 and the paragraph after it): all n_layers*n_heads heads
+ * are ranked by sigma (host, row-major [n_layers][n_heads], already averaged over the samples) and
+ * the round(alpha * n_layers * n_heads) lowest are marked contextual (1), the others structural (0);
+ * equal values rank by (layer, head).  head_is_contextual: host, [n_layers*n_heads], the mask
+ * hack_config_t takes.  Host only.  INVALID_ARG unless 0 <= alpha <= 1 and sigma is finite. */
+HACK_API hack_status_t hack_classify_heads(const double* sigma, int32_t n_layers, int32_t n_heads, double alpha,
+                                  uint8_t* head_is_contextual);
+
 /* The whole step for one (layer, scale): score -> select -> compact -> attend; heads whose
  * candidate count does not exceed their budget skip scoring and selection and keep everything
  * (section "KV Cache Compression for VAR": compress whenever the length exceeds the budget). */

@@ -5,5 +5,5 @@ sources (csrc/), the build script and a ctypes binding with the same names as th
 """
 from .binding import (  # noqa: F401
     HACK_BF16, HACK_F32, HACK_OBS_CALLER, HACK_OBS_INIT, HACK_OBS_RECENT, HACK_OBS_UNIFORM, HACK_OK, HACK_OVERFLOW_COMPETE, HACK_OVERFLOW_KEEP_PROTECTED, RULE_FRACTION,
-    RULE_RATIO, EXPORTS, HackCache, HackError, hack_last_error, hack_score_noalloc, hack_split_budget,
+    RULE_RATIO, EXPORTS, HackCache, HackError, hack_classify_heads, hack_last_error, hack_score_noalloc, hack_split_budget,
 )

@@ -21,7 +21,8 @@ RULE_FRACTION, RULE_RATIO = 0, 1
 
 EXPORTS = (
     "hack_split_budget", "hack_init_cache", "hack_free_cache", "hack_reset", "hack_set_obs_rows", "hack_get_limits",
-    "hack_step_info", "hack_score", "hack_select", "hack_compact", "hack_attend", "hack_scale_step",
+    "hack_step_info", "hack_score", "hack_select", "hack_compact", "hack_attend", "hack_attend_variance",
+    "hack_classify_heads", "hack_scale_step",
     "hack_scale_step_host", "hack_score_noalloc", "hack_get_lengths", "hack_read_head", "hack_kv_bytes",
     "hack_launch_count", "hack_stage_timing", "hack_stage_times", "hack_poll_status", "hack_last_error",
 )
@@ -74,6 +75,8 @@ def _load() -> C.CDLL:
         "hack_select": [vp, i32, i32, vp, vp, vp, vp],
         "hack_compact": [vp, i32, i32, vp, vp, vp, vp],
         "hack_attend": [vp, i32, i32, vp, vp, vp],
+        "hack_attend_variance": [vp, i32, i32, vp, vp, vp, vp],
+        "hack_classify_heads": [C.POINTER(C.c_double), i32, i32, C.c_double, C.POINTER(C.c_uint8)],
         "hack_scale_step": [vp, i32, i32, vp, vp, vp, vp, vp],
         "hack_scale_step_host": [vp, i32, i32, vp, vp, vp, vp, vp],
         "hack_score_noalloc": [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, C.c_float, vp],
@@ -108,6 +111,17 @@ def hack_split_budget(budget: int, alpha: float, rule: int, param: float, total_
     bc, bs = C.c_int32(), C.c_int32()
     _check(lib.hack_split_budget(budget, alpha, rule, param, total_tokens, C.byref(bc), C.byref(bs)))
     return bc.value, bs.value
+
+
+def hack_classify_heads(sigma, n_layers: int, n_heads: int, alpha: float):
+    """Head mask (list of n_layers lists of 0/1, 1 = contextual) from the variance matrix."""
+    flat = [float(v) for row in sigma for v in (row if hasattr(row, "__iter__") else [row])]
+    if len(flat) != n_layers * n_heads:
+        raise ValueError("sigma must have n_layers*n_heads entries")
+    arr = (C.c_double * len(flat))(*flat)
+    out = (C.c_uint8 * len(flat))()
+    _check(lib.hack_classify_heads(arr, n_layers, n_heads, alpha, out))
+    return [[int(out[l * n_heads + h]) for h in range(n_heads)] for l in range(n_layers)]
 
 
 def hack_score_noalloc(q, k_cand, scores, n_rows: int, n_queries: int, n_cand: int, score_stride: int,
@@ -186,6 +200,9 @@ class HackCache:
 
     def hack_attend(self, layer, scale, q, out, stream=None) -> None:
         _check(lib.hack_attend(self._h, layer, scale, _ptr(q), _ptr(out), _ptr(stream)))
+
+    def hack_attend_variance(self, layer, scale, q, out, sigma, stream=None) -> None:
+        _check(lib.hack_attend_variance(self._h, layer, scale, _ptr(q), _ptr(out), _ptr(sigma), _ptr(stream)))
 
     def hack_scale_step(self, layer, scale, q, k, v, out, stream=None) -> None:
         _check(lib.hack_scale_step(self._h, layer, scale, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(stream)))

@@ -58,6 +58,7 @@ struct TcParams {
   const int32_t* row_off;
   const int32_t* head_order;             // longest heads first
   __nv_bfloat16* out;
+  float* row_stats;                      // optional [b*H, N_k, 2]: reference maximum and sum of every softmax row
   int* status;
 };
 
@@ -355,6 +356,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const int row = q0 + t * kBM + r;
         const float inv = 1.f / l;
         __nv_bfloat16* dst = p.out + (static_cast<size_t>(bh) * p.n_new + row) * D;
+        if (p.row_stats && row < p.n_new)
+          *reinterpret_cast<float2*>(p.row_stats + (static_cast<size_t>(bh) * p.n_new + row) * 2) = make_float2(m_used, l);
 #pragma unroll
         for (int ch = 0; ch < D / 32; ++ch) {
           uint32_t orr[32];
@@ -422,7 +425,7 @@ bool make_rows_map(void* out_map, const void* base, uint64_t rows, int head_dim)
 }
 
 int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
-                     const void* q, void* out, cudaStream_t st) {
+                     const void* q, void* out, float* row_stats, cudaStream_t st) {
   CUtensorMap tm_q;
   if (!make_rows_map(&tm_q, q, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) return -1;
   TcParams p;
@@ -439,6 +442,7 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
   p.row_off = a.row_off;
   p.head_order = head_order;
   p.out = static_cast<__nv_bfloat16*>(out);
+  p.row_stats = row_stats;
   p.status = a.status;
   const int grid = p.n_pairs * a.batch * a.n_heads;
   const CUtensorMap& tk = *static_cast<const CUtensorMap*>(k_map);

@@ -27,10 +27,13 @@ void allow_dynamic_smem_impl(const void* kern, size_t bytes) {
   done.emplace_back(kern, dev);
 }
 
-int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st) {
+bool attend_tc_serves(const StepArgs& a, int dtype) {
   // the tensor-core kernel serves bf16 caches once a scale has enough rows for its TMA boxes
-  if (dtype == HACK_BF16 && a.k_map && a.n_new >= kTcMinQueries && (long long)a.batch * a.n_heads * a.n_new >= 128)
-    return launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, st);
+  return dtype == HACK_BF16 && a.k_map && a.n_new >= kTcMinQueries && (long long)a.batch * a.n_heads * a.n_new >= 128;
+}
+
+int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st) {
+  if (attend_tc_serves(a, dtype)) return launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, st);
   return launch_attend_simt(a, dtype, q, out, st);
 }
 
@@ -72,6 +75,9 @@ struct hack_cache {
   hack::Scratch scratch{};
   int* status = nullptr;
   int32_t* n_old = nullptr;                     // [b*H] scratch of the compaction kernels
+  float* attn_row_stats = nullptr;              // bf16 caches: [b*H, max N_k, 2] softmax row statistics (Eq. 6 path)
+  float* attn_block_var = nullptr;              // bf16 caches: [b*H, var_blocks] per key block variances
+  int var_blocks = 0;
   int32_t* obs_rows = nullptr;                  // HACK_OBS_CALLER: [n_scales][kMaxObs] query rows of Q~
   std::vector<uint8_t> obs_rows_set;            // per scale: rows were supplied
   std::vector<TensorMapBox> k_maps, v_maps;     // per layer, bf16 caches only
@@ -398,6 +404,11 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
     HACK_TRY(cudaMemcpy(c->head_order, order.data(), order.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
   }
   HACK_TRY(cudaMalloc(&c->n_old, (size_t)bh * sizeof(int32_t)));
+  if (cfg->dtype == HACK_BF16) {
+    c->var_blocks = c->limits.kept_stride / 128 + 1;
+    HACK_TRY(cudaMalloc(&c->attn_row_stats, (size_t)bh * c->limits.max_new * 2 * sizeof(float)));
+    HACK_TRY(cudaMalloc(&c->attn_block_var, (size_t)bh * c->var_blocks * sizeof(float)));
+  }
   if (cfg->obs_sampler == HACK_OBS_CALLER) {
     HACK_TRY(cudaMalloc(&c->obs_rows, (size_t)cfg->n_scales * hack::kMaxObs * sizeof(int32_t)));
     HACK_TRY(cudaMemset(c->obs_rows, 0, (size_t)cfg->n_scales * hack::kMaxObs * sizeof(int32_t)));
@@ -420,6 +431,8 @@ hack_status_t hack_free_cache(hack_cache_t* c) {
   cudaFree(c->scratch.logits); cudaFree(c->scratch.partials); cudaFree(c->status);
   cudaFree(c->head_order);
   cudaFree(c->n_old);
+  cudaFree(c->attn_row_stats);
+  cudaFree(c->attn_block_var);
   cudaFree(c->obs_rows);
   for (int sl = 0; sl < hack_cache::kHostSlots; ++sl) {
     for (int i = 0; i < 4; ++i) cudaFree(c->stage[sl][i]);
@@ -528,7 +541,8 @@ hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const 
   return HACK_OK;
 }
 
-static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void* q, void* out, cudaStream_t st) {
+static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void* q, void* out, float* sigma,
+                                 cudaStream_t st) {
   // lengths are already those after compaction
   LayerState& ls = c->layers[layer];
   hack_step_info_t p{};
@@ -538,7 +552,19 @@ static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void
   p.n_obs_rows = std::min(c->cfg.n_obs, p.n_new);
   const hack::StepArgs a = make_args(c, layer, scale, p);
   StageScope ts(c, st, 3);
-  const int n = hack::launch_attend(a, c->cfg.dtype, q, out, st);
+  int n;
+  if (sigma) {
+    // Eq. 6 needs the statistics of every softmax row; the tensor-core attention kernel leaves them
+    if (!hack::attend_tc_serves(a, c->cfg.dtype))
+      return fail(HACK_ERR_UNSUPPORTED, "hack_attend_variance needs a bf16 cache and a scale of at least 32 tokens (128 query rows over all heads)");
+    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, c->attn_row_stats, st);
+    if (n >= 0) {
+      const int m = hack::launch_attention_variance(a, q, c->attn_row_stats, c->attn_block_var, c->var_blocks, sigma, st);
+      n = m < 0 ? m : n + m;
+    }
+  } else {
+    n = hack::launch_attend(a, c->cfg.dtype, q, out, st);
+  }
   if (n < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
   ts.done(n);
   c->launches += n;
@@ -552,7 +578,33 @@ hack_status_t hack_attend(hack_cache_t* c, int32_t layer, int32_t scale, const v
   if (s != HACK_OK) return s;
   if (!q || !out) return fail(HACK_ERR_INVALID_ARG, "q or out is NULL");
   if (misaligned(q) || misaligned(out)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
-  return attend_impl(c, layer, scale, q, out, (cudaStream_t)stream);
+  return attend_impl(c, layer, scale, q, out, nullptr, (cudaStream_t)stream);
+}
+
+hack_status_t hack_attend_variance(hack_cache_t* c, int32_t layer, int32_t scale, const void* q, void* out,
+                                   float* sigma, void* stream) {
+  hack_status_t s = check_step(c, layer, scale, 1);
+  if (s != HACK_OK) return s;
+  if (!q || !out || !sigma) return fail(HACK_ERR_INVALID_ARG, "q, out or sigma is NULL");
+  if (misaligned(q) || misaligned(out)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
+  return attend_impl(c, layer, scale, q, out, sigma, (cudaStream_t)stream);
+}
+
+hack_status_t hack_classify_heads(const double* sigma, int32_t n_layers, int32_t n_heads, double alpha,
+                                  uint8_t* head_is_contextual) {
+  if (!sigma || !head_is_contextual) return fail(HACK_ERR_INVALID_ARG, "sigma or head_is_contextual is NULL");
+  if (n_layers < 1 || n_heads < 1) return fail(HACK_ERR_INVALID_ARG, "n_layers and n_heads must be positive");
+  if (!(alpha >= 0.0 && alpha <= 1.0)) return fail(HACK_ERR_INVALID_ARG, "alpha must be in [0, 1]");
+  const int n = n_layers * n_heads;
+  for (int i = 0; i < n; ++i)
+    if (!std::isfinite(sigma[i])) return fail(HACK_ERR_INVALID_ARG, "sigma must be finite");
+  std::vector<int> order(n);
+  for (int i = 0; i < n; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int x, int y) { return sigma[x] < sigma[y]; });
+  const int n_ctx = (int)std::floor(alpha * n + 0.5);
+  for (int i = 0; i < n; ++i) head_is_contextual[i] = 0;
+  for (int i = 0; i < n_ctx; ++i) head_is_contextual[order[i]] = 1;
+  return HACK_OK;
 }
 
 hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, const void* q,
@@ -603,7 +655,7 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
   }
   c->launches += n;
   advance_after_compact(c, layer, p);
-  return attend_impl(c, layer, scale, q, out, st);
+  return attend_impl(c, layer, scale, q, out, nullptr, st);
 }
 
 hack_status_t hack_scale_step_host(hack_cache_t* c, int32_t layer, int32_t scale, const void* q_host,

@@ -66,8 +66,15 @@ int launch_compact(const StepArgs& a, int dtype, const int32_t* idx, int idx_all
 int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st);
 
 int launch_attend_simt(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st);
+// row_stats (optional, device [b*H, N_k, 2]): per query row the reference maximum m (raw logit
+// units; within the lazy-rescaling margin of the true maximum) and l = sum_j exp2(c (z_j - m)).
 int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
-                     const void* q, void* out, cudaStream_t st);
+                     const void* q, void* out, float* row_stats, cudaStream_t st);
+// Attention variance per (batch, head) over the compacted cache (Eq. 6) from the row statistics of
+// launch_attend_tc; block_var: device scratch [b*H, max_blocks]; sigma: device [b*H].  bf16 only.
+int launch_attention_variance(const StepArgs& a, const void* q, const float* row_stats, float* block_var,
+                              int max_blocks, float* sigma, cudaStream_t st);
+bool attend_tc_serves(const StepArgs& a, int dtype);   // the tensor-core kernel takes this step's attention
 // 2-D bf16 tensor map (128 x 64 boxes, 128-byte swizzle) over rows x head_dim; false on failure.
 bool make_rows_map(void* out_map, const void* base, uint64_t rows, int head_dim);
 

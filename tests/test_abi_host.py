@@ -86,3 +86,19 @@ def test_product_package_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".h", ".cuh")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.lower(), f
+
+
+def test_classify_heads_matches_the_oracle_rule(hb):
+    import numpy as np
+    from oracle import hack_oracle as ho
+    assert hb.hack_classify_heads([[0.9, 0.1, 0.5], [0.2, 0.8, 0.1]], 2, 3, 0.5) == [[0, 1, 0], [1, 0, 1]]
+    assert hb.hack_classify_heads([[0.0, 0.0], [0.0, 0.0]], 2, 2, 0.5) == [[1, 1], [0, 0]]      # ties: (layer, head) order
+    rng = np.random.default_rng(11)
+    for alpha in (0.0, 0.25, 0.4, 0.5, 0.75, 1.0):
+        sigma = rng.lognormal(size=(5, 7))
+        sigma[2, 3] = sigma[0, 1]                                                              # a tie across layers
+        assert hb.hack_classify_heads(sigma.tolist(), 5, 7, alpha) == ho.classify_heads(sigma, alpha).tolist()
+    for bad in (([[0.1, float("nan")]], 1, 2, 0.5), ([[0.1, 0.2]], 1, 2, 1.5), ([[0.1, 0.2]], 1, 2, -0.1)):
+        with pytest.raises(hb.HackError) as e:
+            hb.hack_classify_heads(*bad)
+        assert e.value.status == 1

@@ -496,6 +496,85 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_head_variance(args):
+    """Separate measurement (not part of the decoding loop): the attention-variance pass of the offline
+    head classification (Eq. 6) on one layer of the chosen workload, uncompressed cache, last scale.
+    Prints its own JSON line.  The pass evaluates one exponential per (query, key) pair, so it is
+    bound by the special-function units: 16 exp2 per clock and SM."""
+    import torch
+    import paper_2504_09261_b200 as hb
+    from workloads import SyntheticQKV, get_config
+    cfg = get_config(args.config, n_layers=1)
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    gen = SyntheticQKV(cfg, device=dev)
+    mask = gen.head_is_contextual
+    t_k = cfg.total_tokens
+    K = cfg.n_scales
+    bh = cfg.batch * cfg.n_heads
+    cache = hb.HackCache(1, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides, hb.HACK_BF16, mask.numpy(), t_k, t_k,
+                         n_obs=cfg.n_obs, device=0)
+    qkv = [gen.qkv(0, k) for k in range(K)]
+    outs = [torch.empty_like(qkv[k][0]) for k in range(K)]
+    scores = torch.empty((bh, cache.cand_stride), dtype=torch.float32, device=dev)
+    idx = torch.empty((bh, cache.kept_stride), dtype=torch.int32, device=dev)
+    sigma = torch.zeros(bh, device=dev)
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+
+    def one(with_variance):
+        cache.hack_reset()
+        for k in range(K - 1):
+            q, kk, v = qkv[k]
+            cache.hack_scale_step(0, k, q, kk, v, outs[k], sh)
+        q, kk, v = qkv[K - 1]
+        cache.hack_score(0, K - 1, q, kk, scores, sh)
+        cache.hack_select(0, K - 1, scores, idx, None, sh)
+        cache.hack_compact(0, K - 1, idx, kk, v, sh)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        if with_variance:
+            cache.hack_attend_variance(0, K - 1, q, outs[K - 1], sigma, sh)
+        else:
+            cache.hack_attend(0, K - 1, q, outs[K - 1], sh)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        one(True)
+        one(False)
+    both = sorted(one(True) for _ in range(max(args.steps, 5)))
+    plain = sorted(one(False) for _ in range(max(args.steps, 5)))
+    clocks = sampler.stop()
+    ms_both, ms_plain = both[len(both) // 2], plain[len(plain) // 2]
+    ms_var = ms_both - ms_plain
+    n_k = cfg.tokens_per_scale[-1]
+    pairs = float(bh) * n_k * t_k
+    props = torch.cuda.get_device_properties(0)
+    sm_mhz = clocks.get("sm_max_mhz") or 1965.0
+    peak = 16.0 * props.multi_processor_count * sm_mhz * 1e6
+    print(json.dumps({
+        "metric": "attention-variance pass of the offline head classification (Eq. 6), (query, key) pairs per second",
+        "value": pairs / (ms_var * 1e-3), "unit": "pairs/s", "n_gpus": 1, "higher_is_better": True,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"config {args.config}, one layer, uncompressed cache, last scale: "
+                               f"{bh} heads x {n_k} queries x {t_k} keys, head_dim {cfg.head_dim}"},
+        "ms_attend": ms_plain, "ms_attend_with_variance": ms_both, "ms_variance_kernels": ms_var,
+        "roofline": {"kernel": "attn_colstats_kernel", "bound": "alu", "achieved": pairs / (ms_var * 1e-3) / 1e9,
+                     "peak": peak / 1e9, "unit": "G exp2/s", "frac": pairs / (ms_var * 1e-3) / peak,
+                     "peak_source": f"16 exp2 per clock and SM x {props.multi_processor_count} SMs x {sm_mhz:.0f} MHz (clocks.max.sm)",
+                     "traffic": None},
+        "tensor_tflops": 2.0 * pairs * cfg.head_dim / (ms_var * 1e-3) / 1e12,
+        "sigma_mean_contextual": float(sigma.view(cfg.batch, cfg.n_heads)[:, mask[0].bool()].mean()),
+        "sigma_mean_structural": float(sigma.view(cfg.batch, cfg.n_heads)[:, ~mask[0].bool()].mean()),
+        "clocks": clocks,
+    }))
+    cache.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -509,9 +588,13 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--head-variance", action="store_true",
+                    help="time the attention-variance pass of the offline head classification instead of the loop")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    if args.head_variance:
+        run_head_variance(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -9,7 +9,7 @@
 //   warp 1    : tcgen05.mma issuer; S^T = K_blk Q_tile^T, keys on the 128 TMEM lanes, queries on
 //               128 columns, two accumulators so that the next MMA runs under the current read-out
 //   warps 2-5 : consumers; thread r owns key r: it reads its 128 logits with tcgen05.ld, forms
-//               p = exp2(c z - c m_i) / l_i and adds p and p^2 to two registers
+//               p = exp2(c z - c m_i - log2 l_i) and adds p and p^2 to two registers
 // so the sums over the queries stay inside one thread and nothing of size N x T is stored.  At the
 // end the thread holds Var_i A[i, j] = sum p^2 / N - (sum p / N)^2 of its key; the CTA adds its 128
 // variances and a second, tiny kernel adds the blocks of a head in a fixed order.
@@ -79,7 +79,7 @@ attn_colstats_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   const uint32_t k_sm = base;
   const uint32_t q_sm = base + TILE_BYTES;
   VarBars* bars = reinterpret_cast<VarBars*>(sm + (1 + kQStages) * TILE_BYTES);
-  __shared__ float2 stat[2][kVarTile];           // (-c m_i, 1 / l_i) of the query tile in accumulator b
+  __shared__ __align__(16) float stat[2][kVarTile];   // -c m_i - log2 l_i of the query tile in accumulator b
   __shared__ float red[4];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -168,10 +168,10 @@ attn_colstats_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       {
         // statistics of query ct of this tile; queries past the end of the scale get weight 0
         const int qi = t * kVarTile + ct;
-        float2 st = make_float2(0.f, 0.f);
+        float st = -INFINITY;                      // exp2(-inf) = 0
         if (qi < a.n_new) {
           const float2 ml = *reinterpret_cast<const float2*>(row_stats + ((size_t)bh * a.n_new + qi) * 2);
-          st = make_float2(-ml.x * c, 1.f / ml.y);
+          st = -ml.x * c - __log2f(ml.y);          // p = exp2(c z - c m - log2 l): the division is in the exponent
         }
         stat[b][ct] = st;
       }
@@ -189,17 +189,19 @@ attn_colstats_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
           mbar_arrive(smem_u32(&bars->acc_free[b]));
         }
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float2 st = stat[b][ch * 32 + i];
-          // a query of another head (or a zero row past the tensor's end) has weight 0; its logit
-          // may be large, so the exponent is capped to keep the product finite
-          const float p = ex2(fminf(fmaf(__uint_as_float(acc[i]), c, st.x), 64.f)) * st.y;
-          sum_p += p;
-          sum_p2 = fmaf(p, p, sum_p2);
+        for (int i = 0; i < 32; i += 4) {
+          const float4 st = *reinterpret_cast<const float4*>(&stat[b][ch * 32 + i]);
+          const float p0 = ex2(fmaf(__uint_as_float(acc[i]), c, st.x));
+          const float p1 = ex2(fmaf(__uint_as_float(acc[i + 1]), c, st.y));
+          const float p2 = ex2(fmaf(__uint_as_float(acc[i + 2]), c, st.z));
+          const float p3 = ex2(fmaf(__uint_as_float(acc[i + 3]), c, st.w));
+          sum_p += (p0 + p1) + (p2 + p3);
+          sum_p2 = fmaf(p0, p0, fmaf(p1, p1, fmaf(p2, p2, fmaf(p3, p3, sum_p2))));
         }
       }
     }
-    // Var_i A[i, j] of this thread's key; keys past the end of the head count nothing
+    // Var_i A[i, j] of this thread's key; keys past the end of the head count nothing (their sums
+    // come from rows of another head and may have overflowed)
     const float inv_n = 1.f / (float)a.n_new;
     float var = 0.f;
     if (ok && kb * kVarTile + key_row < len) {

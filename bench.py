@@ -208,9 +208,10 @@ def run_ours(args):
     n_ctx = [int(mask[l].sum()) for l in range(L)]
     dtype_id = hb.HACK_F32 if cfg.dtype == "f32" else hb.HACK_BF16
 
-    def new_cache(bc, bs):
+    def new_cache(bc, bs, policy=0):
         return hb.HackCache(L, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides, dtype_id, mask.numpy(),
-                            bc, bs, n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, device=local)
+                            bc, bs, n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, overflow_policy=policy,
+                            device=local)
 
     cache = new_cache(cfg.budget_c, cfg.budget_s)
     # inputs resident in HBM: every (layer, scale) has its own Q, K, V (ranks draw different images)
@@ -296,6 +297,48 @@ def run_ours(args):
         return ms, scale_ms
 
     use_graph = not args.no_graph
+    if args.latency_profile:
+        # Attention-module latency per scale (score + select + compact + attend of every layer) for the
+        # uncompressed cache and for compression ratios rho = 1 - B / T_K, budgets split 1 : 2 between
+        # contextual and structural heads (Eq. 7).  The cumulative time up to the scale whose side is
+        # 16 / 32 / 64 is the latency of a 256 / 512 / 1024 pixel image under this schedule: the
+        # resolution axis of the paper's latency profile.  One JSON line.
+        cache.close()
+        t_k = cfg.total_tokens
+        rows = []
+        for rho, policy in ((0.0, 0), (0.3, 0), (0.5, 0), (0.7, 0), (0.9, 0), (0.9, 1)):
+            if rho == 0.0:
+                bc = bs = t_k
+            else:
+                bc, bs = hb.hack_split_budget(int((1.0 - rho) * t_k + 1e-9), cfg.alpha, hb.RULE_RATIO, 2.0, t_k)
+            c = new_cache(bc, bs, policy)
+            ms, scale_ms = timed(c, args.steps, args.warmup, per_scale=True, use_graph=use_graph)
+            _, peak_kv, _ = c.hack_kv_bytes()
+            c.close()
+            cum = 0.0
+            at_side = {}
+            for k in range(K):
+                cum += scale_ms[k]
+                at_side[cfg.sides[k]] = cum
+            rows.append({"rho": rho, "budget_c": bc, "budget_s": bs,
+                         "overflow_policy": "keep protected" if policy == 0 else "compete",
+                         "ms_per_image_batch": ms / args.steps, "ms_per_scale": [round(x, 4) for x in scale_ms],
+                         "ms_up_to_side": {str(sd): round(at_side[sd], 4) for sd in (16, 32, 64) if sd in at_side},
+                         "peak_kv_bytes": peak_kv})
+        full = rows[0]
+        for r in rows:
+            r["speedup_vs_full"] = full["ms_per_image_batch"] / r["ms_per_image_batch"]
+            r["speedup_last_scale"] = full["ms_per_scale"][-1] / r["ms_per_scale"][-1]
+        if rank == 0:
+            print(json.dumps({"metric": "attention-module latency per scale, uncompressed against compressed",
+                              "unit": "ms", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                              "dtype": cfg.dtype, "data": "synthetic",
+                              "config": {"workload": cfg.name, "layers": L, "sides": list(cfg.sides),
+                                         "timing": "CUDA graph replay" if use_graph else "direct calls"},
+                              "rows": rows}))
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     launches0 = cache.hack_launch_count()
     loop(cache)
     launches_per_step = cache.hack_launch_count() - launches0
@@ -588,6 +631,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--latency-profile", action="store_true",
+                    help="per-scale latency of the uncompressed cache and of compression ratios 30-90 %% instead of the loop")
     ap.add_argument("--head-variance", action="store_true",
                     help="time the attention-variance pass of the offline head classification instead of the loop")
     args = ap.parse_args()

@@ -13,6 +13,9 @@ the tests, the smoke check and the CPU-baseline leg of the benchmark may use it.
 Parity pins (see tests/test_oracle_*.py): full-budget == vanilla attention (Eq. 3-4), softmax
 row sums, brute-force subset selection, protected-scale invariants, the closed forms of the
 complexity analysis (Eq. 12-22), convexity and permutation invariance of the attention output.
+The final-scale merge of contextual heads (merge_assign, merge_apply) follows one sentence of the
+paper; the similarity measure, the weights and the treatment of V are a reading: parity unpinned
+(pins cover only what the reading itself fixes: special cases, an explicit loop, convexity).
 Offline head classification (Eq. 6) is here too: attention_variance and classify_heads, pinned by
 closed forms (identity and uniform attention) and by recovering a planted head mask.
 Parity unpinned (the paper is silent; only self-consistency is tested): the overflow rule when
@@ -127,6 +130,39 @@ def attend(q: np.ndarray, k_hat: np.ndarray, v_hat: np.ndarray, sm_scale: float)
     return softmax_rows(sm_scale * (q @ k_hat.T)) @ v_hat
 
 
+# --------------------------------------------------------------------------- final-scale merge
+def merge_assign(k_evicted: np.ndarray, k_kept: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Nearest retained counterpart of every discarded key, and its weight.
+
+    The paper gives the merge one sentence (contextual-head strategy, after Eq. 10): discarded KV
+    tokens of the last step are folded into their nearest retained counterparts by similarity-weighted
+    averaging.  Reading taken here (the paper is silent on all three points): nearness is the cosine
+    similarity between keys; the counterpart is the retained key with the largest similarity, the
+    lowest index among equals; the weight is that similarity, or 0 if it is negative.
+    Returns (index into the kept list, weight) per discarded entry."""
+    ne = np.linalg.norm(k_evicted, axis=1, keepdims=True)
+    nk = np.linalg.norm(k_kept, axis=1, keepdims=True)
+    cos = (k_evicted @ k_kept.T) / np.maximum(ne * nk.T, 1e-300)
+    assign = np.argmax(cos, axis=1).astype(np.int64)
+    weight = np.maximum(cos[np.arange(cos.shape[0]), assign], 0.0)
+    return assign, weight
+
+
+def merge_apply(k_kept: np.ndarray, v_kept: np.ndarray, k_evicted: np.ndarray, v_evicted: np.ndarray,
+                assign: np.ndarray, weight: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Similarity-weighted average of every retained entry with the discarded entries assigned to it:
+    k_c <- (k_c + sum_e w_e k_e) / (1 + sum_e w_e), the same weights for v_c (the retained entry
+    itself has similarity 1).  Entries without assignments are unchanged."""
+    num_k, num_v = k_kept.copy(), v_kept.copy()
+    den = np.ones(k_kept.shape[0])
+    for e in range(k_evicted.shape[0]):
+        c = int(assign[e])
+        num_k[c] += weight[e] * k_evicted[e]
+        num_v[c] += weight[e] * v_evicted[e]
+        den[c] += weight[e]
+    return num_k / den[:, None], num_v / den[:, None]
+
+
 # --------------------------------------------------------------------------- state
 @dataclass
 class HeadCache:
@@ -144,6 +180,9 @@ class StepRecord:
     scores: Optional[np.ndarray]      # fp64 scores the oracle computed (None if not triggered)
     keep: np.ndarray                  # ascending candidate indices that survive
     pos: np.ndarray                   # their global token positions
+    evicted: Optional[np.ndarray] = None        # final-scale merge: ascending candidate indices discarded
+    merge_assign: Optional[np.ndarray] = None   # ... index into `keep` each of them was folded into
+    merge_weight: Optional[np.ndarray] = None   # ... and its weight
 
 
 @dataclass
@@ -161,7 +200,8 @@ class HackOracle:
                  sides: Sequence[int], head_is_contextual: np.ndarray,
                  budget_c: int, budget_s: int, n_obs: int = 32, n_init_scales: int = 2,
                  sm_scale: Optional[float] = None, overflow_policy: int = KEEP_PROTECTED,
-                 obs_sampler: int = UNIFORM, obs_rows: Optional[Sequence[Sequence[int]]] = None):
+                 obs_sampler: int = UNIFORM, obs_rows: Optional[Sequence[Sequence[int]]] = None,
+                 merge_last: bool = False):
         self.L, self.H, self.b, self.D = n_layers, n_heads, batch, head_dim
         self.sides = tuple(int(s) for s in sides)
         self.N = tuple(s * s for s in self.sides)
@@ -173,6 +213,7 @@ class HackOracle:
         self.policy = overflow_policy
         self.obs_sampler = obs_sampler
         self.obs_rows = obs_rows            # CALLER: one row list per scale
+        self.merge_last = bool(merge_last)  # contextual heads fold what the last scale evicts into what it keeps
         self.counters = Counters()
         self.reset()
 
@@ -194,11 +235,15 @@ class HackOracle:
     # ----------------------------------------------------------------------- one head
     def head_step(self, layer: int, scale: int, b: int, h: int, q: np.ndarray, k_new: np.ndarray,
                   v_new: np.ndarray, scores_override: Optional[np.ndarray] = None,
-                  need_output: bool = True) -> Tuple[Optional[np.ndarray], StepRecord]:
+                  need_output: bool = True,
+                  assign_override: Optional[np.ndarray] = None) -> Tuple[Optional[np.ndarray], StepRecord]:
         """One (batch, head) of one step.  `scale` is 0-based here, the paper's k is scale + 1.
 
         scores_override: fp32/fp64 scores over the candidates to be used for the selection in
         place of the oracle's own (teacher forcing, so near-ties cannot cascade).
+        assign_override: with the final-scale merge, the counterpart of every discarded entry to be
+        used in place of the oracle's own argmax (same reason); the weights are then the similarities
+        to those counterparts.
         """
         k1 = scale + 1
         n_k = self.N[scale]
@@ -232,12 +277,26 @@ class HackOracle:
         # 3. gather survivors in ascending position
         self._live += keep.shape[0] - st.k.shape[0]
         st.k, st.v, st.pos, st.sid = k_c[keep], v_c[keep], pos_c[keep], sid_c[keep]
+        # 3b. only at the final scale, only in contextual heads: fold the discarded entries of this
+        # step into their nearest retained counterparts
+        evicted = m_assign = m_weight = None
+        if self.merge_last and compressed and scale == len(self.N) - 1 and self.is_ctx[layer, h]:
+            gone = np.ones(t_cand, dtype=bool)
+            gone[keep] = False
+            evicted = np.nonzero(gone)[0]
+            m_assign, m_weight = merge_assign(k_c[evicted], st.k)
+            if assign_override is not None:
+                m_assign = np.asarray(assign_override, dtype=np.int64)
+                ke, kk = k_c[evicted], st.k[m_assign]
+                cos = (ke * kk).sum(axis=1) / np.maximum(np.linalg.norm(ke, axis=1) * np.linalg.norm(kk, axis=1), 1e-300)
+                m_weight = np.maximum(cos, 0.0)
+            st.k, st.v = merge_apply(st.k, st.v, k_c[evicted], v_c[evicted], m_assign, m_weight)
         # 4. attention of all N_k queries over the compressed cache
         out = None
         if need_output:
             out = attend(q, st.k, st.v, self.sm_scale)
         self.counters.attention_pairs += n_k * keep.shape[0]
-        return out, StepRecord(compressed, t_cand, scores, keep, st.pos.copy())
+        return out, StepRecord(compressed, t_cand, scores, keep, st.pos.copy(), evicted, m_assign, m_weight)
 
     # ----------------------------------------------------------------------- all heads
     def scale_step(self, layer: int, scale: int, q: np.ndarray, k: np.ndarray, v: np.ndarray,

@@ -447,3 +447,72 @@ def test_variance_ranking_recovers_the_planted_head_types():
     alpha = float(mask.mean())
     assert ho.classify_heads(sigma, alpha).tolist() == mask.tolist()
     assert sigma[mask == 1].max() < sigma[mask == 0].min()
+
+
+# ------------------------------------------------------------------ final-scale merge (a reading; see the oracle's header)
+def test_merge_special_cases():
+    """What the reading fixes by itself: a discarded entry identical to a retained one is averaged in
+    with weight 1; one orthogonal or opposed to every retained key changes nothing; retained entries
+    without assignments keep their bits; equal similarities go to the lowest index."""
+    k_kept = np.array([[1.0, 0.0, 0.0], [0.0, 2.0, 0.0], [0.0, 2.0, 0.0]])
+    v_kept = np.array([[1.0, 1.0, 1.0], [2.0, 2.0, 2.0], [3.0, 3.0, 3.0]])
+    k_ev = np.array([[3.0, 0.0, 0.0], [0.0, 0.0, 5.0], [-1.0, -1.0, 0.0], [0.0, 1.0, 0.0]])
+    v_ev = np.array([[5.0, 5.0, 5.0], [9.0, 9.0, 9.0], [7.0, 7.0, 7.0], [4.0, 4.0, 4.0]])
+    assign, weight = ho.merge_assign(k_ev, k_kept)
+    assert assign.tolist()[0] == 0 and weight[0] == pytest.approx(1.0)
+    assert weight[1] == 0.0 and weight[2] == 0.0
+    assert assign.tolist()[3] == 1 and weight[3] == pytest.approx(1.0)       # tie between kept 1 and 2: lowest index
+    k_m, v_m = ho.merge_apply(k_kept, v_kept, k_ev, v_ev, assign, weight)
+    np.testing.assert_allclose(k_m[0], [2.0, 0.0, 0.0])                      # (k_c + 1 * k_e) / 2
+    np.testing.assert_allclose(v_m[0], [3.0, 3.0, 3.0])
+    np.testing.assert_allclose(k_m[1], [0.0, 1.5, 0.0])
+    np.testing.assert_allclose(v_m[1], [3.0, 3.0, 3.0])
+    assert np.array_equal(k_m[2], k_kept[2]) and np.array_equal(v_m[2], v_kept[2])
+
+
+def test_merge_matches_loops_and_stays_in_the_hull():
+    rng = np.random.default_rng(8)
+    k_kept, v_kept = rng.normal(size=(6, 5)), rng.normal(size=(6, 5))
+    k_ev, v_ev = rng.normal(size=(11, 5)), rng.normal(size=(11, 5))
+    assign, weight = ho.merge_assign(k_ev, k_kept)
+    k_m, v_m = ho.merge_apply(k_kept, v_kept, k_ev, v_ev, assign, weight)
+    for c in range(6):
+        num_k, num_v, den = list(k_kept[c]), list(v_kept[c]), 1.0
+        for e in range(11):
+            best, best_c = -2.0, -1
+            for cc in range(6):
+                dot = sum(k_ev[e, t] * k_kept[cc, t] for t in range(5))
+                cos = dot / math.sqrt(sum(x * x for x in k_ev[e]) * sum(x * x for x in k_kept[cc]))
+                if cos > best:
+                    best, best_c = cos, cc
+            if best_c == c and best > 0:
+                for t in range(5):
+                    num_k[t] += best * k_ev[e, t]
+                    num_v[t] += best * v_ev[e, t]
+                den += best
+        np.testing.assert_allclose(k_m[c], np.array(num_k) / den, rtol=1e-12)
+        np.testing.assert_allclose(v_m[c], np.array(num_v) / den, rtol=1e-12)
+    both = np.concatenate([v_kept, v_ev])
+    assert np.all(v_m >= both.min(axis=0) - 1e-12) and np.all(v_m <= both.max(axis=0) + 1e-12)
+
+
+def test_merge_runs_only_at_the_last_scale_of_contextual_heads():
+    rng = np.random.default_rng(9)
+    sides, D = (1, 2, 3, 4), 8
+    mask = np.array([[1, 0]])
+    plain = ho.HackOracle(1, 2, 1, D, sides, mask, budget_c=6, budget_s=30)
+    merged = ho.HackOracle(1, 2, 1, D, sides, mask, budget_c=6, budget_s=30, merge_last=True)
+    for k, side in enumerate(sides):
+        n = side * side
+        q, kk, v = (rng.normal(size=(1, 2, n, D)) for _ in range(3))
+        o_p, rec_p = plain.scale_step(0, k, q, kk, v)
+        o_m, rec_m = merged.scale_step(0, k, q, kk, v)
+        last = k == len(sides) - 1
+        assert (rec_m[(0, 0)].merge_assign is not None) == last and rec_m[(0, 1)].merge_assign is None
+        assert np.array_equal(rec_p[(0, 0)].keep, rec_m[(0, 0)].keep)           # the selection is the same
+        if last:
+            rec = rec_m[(0, 0)]
+            assert len(rec.evicted) + len(rec.keep) == rec.n_candidates
+            assert not np.allclose(o_p[0, 0], o_m[0, 0]) and np.array_equal(o_p[0, 1], o_m[0, 1])
+        else:
+            assert np.array_equal(o_p, o_m)

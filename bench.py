@@ -211,7 +211,7 @@ def run_ours(args):
     def new_cache(bc, bs, policy=0):
         return hb.HackCache(L, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides, dtype_id, mask.numpy(),
                             bc, bs, n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, overflow_policy=policy,
-                            device=local)
+                            device=local, merge_last=args.merge_last)
 
     cache = new_cache(cfg.budget_c, cfg.budget_s)
     # inputs resident in HBM: every (layer, scale) has its own Q, K, V (ranks draw different images)
@@ -631,6 +631,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--merge-last", action="store_true",
+                    help="contextual heads fold what the last scale discards into what it keeps (off in the paper's efficiency runs' default here)")
     ap.add_argument("--latency-profile", action="store_true",
                     help="per-scale latency of the uncompressed cache and of compression ratios 30-90 %% instead of the loop")
     ap.add_argument("--head-variance", action="store_true",

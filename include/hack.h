@@ -84,6 +84,9 @@ typedef struct {
   int32_t overflow_policy;           /* HACK_OVERFLOW_* */
   int32_t device;                    /* CUDA device ordinal */
   int32_t obs_sampler;               /* HACK_OBS_*; 0 = the method's uniform rule */
+  int32_t merge_last;                /* 1: at the last scale, contextual heads fold the entries that step
+                                        discards into their nearest retained counterparts (the merge
+                                        described after Eq. 10; see hack_compact).  bf16 caches only. */
 } hack_config_t;
 
 /* Host-side plan of one step of one layer (all lengths in entries per head). */
@@ -153,7 +156,13 @@ HACK_API hack_status_t hack_select(hack_cache_t* cache, int32_t layer, int32_t s
 
 /* Gather the surviving K/V rows (Eq. 10-11) into the layer's ragged cache in ascending original
  * position; evicted entries are gone for good.  `idx` as written by hack_select for this step;
- * each head's row must hold exactly hack_step_info's kept_c / kept_s entries.  In place. */
+ * each head's row must hold exactly hack_step_info's kept_c / kept_s entries.  In place.
+ * With merge_last, at the last scale, a contextual head that evicts then folds every discarded
+ * entry e into the retained entry c whose key has the largest cosine similarity to k_e (lowest
+ * index among equals) with weight w_e = max(similarity, 0):
+ *   k_c <- (k_c + sum w_e k_e) / (1 + sum w_e), v_c likewise, rounded to bf16
+ * (the paper states the operation in one sentence; measure, weights and the treatment of V are this
+ * library's reading).  hack_scale_step does the same. */
 HACK_API hack_status_t hack_compact(hack_cache_t* cache, int32_t layer, int32_t scale, const int32_t* idx,
                            const void* k_new, const void* v_new, void* stream);
 

@@ -183,6 +183,10 @@ class StepRecord:
     evicted: Optional[np.ndarray] = None        # final-scale merge: ascending candidate indices discarded
     merge_assign: Optional[np.ndarray] = None   # ... index into `keep` each of them was folded into
     merge_weight: Optional[np.ndarray] = None   # ... and its weight
+    evicted_k: Optional[np.ndarray] = None      # ... the discarded rows themselves
+    evicted_v: Optional[np.ndarray] = None
+    kept_k_before: Optional[np.ndarray] = None  # ... and the retained rows before the fold
+    kept_v_before: Optional[np.ndarray] = None
 
 
 @dataclass
@@ -279,7 +283,7 @@ class HackOracle:
         st.k, st.v, st.pos, st.sid = k_c[keep], v_c[keep], pos_c[keep], sid_c[keep]
         # 3b. only at the final scale, only in contextual heads: fold the discarded entries of this
         # step into their nearest retained counterparts
-        evicted = m_assign = m_weight = None
+        evicted = m_assign = m_weight = ev_k = ev_v = kk_before = kv_before = None
         if self.merge_last and compressed and scale == len(self.N) - 1 and self.is_ctx[layer, h]:
             gone = np.ones(t_cand, dtype=bool)
             gone[keep] = False
@@ -290,13 +294,15 @@ class HackOracle:
                 ke, kk = k_c[evicted], st.k[m_assign]
                 cos = (ke * kk).sum(axis=1) / np.maximum(np.linalg.norm(ke, axis=1) * np.linalg.norm(kk, axis=1), 1e-300)
                 m_weight = np.maximum(cos, 0.0)
-            st.k, st.v = merge_apply(st.k, st.v, k_c[evicted], v_c[evicted], m_assign, m_weight)
+            ev_k, ev_v, kk_before, kv_before = k_c[evicted], v_c[evicted], st.k, st.v
+            st.k, st.v = merge_apply(st.k, st.v, ev_k, ev_v, m_assign, m_weight)
         # 4. attention of all N_k queries over the compressed cache
         out = None
         if need_output:
             out = attend(q, st.k, st.v, self.sm_scale)
         self.counters.attention_pairs += n_k * keep.shape[0]
-        return out, StepRecord(compressed, t_cand, scores, keep, st.pos.copy(), evicted, m_assign, m_weight)
+        return out, StepRecord(compressed, t_cand, scores, keep, st.pos.copy(), evicted, m_assign, m_weight,
+                               ev_k, ev_v, kk_before, kv_before)
 
     # ----------------------------------------------------------------------- all heads
     def scale_step(self, layer: int, scale: int, q: np.ndarray, k: np.ndarray, v: np.ndarray,

@@ -35,6 +35,7 @@ class HackConfig(C.Structure):
         ("head_is_contextual", C.POINTER(C.c_uint8)), ("budget_c", C.c_int32), ("budget_s", C.c_int32),
         ("n_obs", C.c_int32), ("n_init_scales", C.c_int32), ("sm_scale", C.c_float),
         ("overflow_policy", C.c_int32), ("device", C.c_int32), ("obs_sampler", C.c_int32),
+        ("merge_last", C.c_int32),
     ]
 
 
@@ -147,7 +148,7 @@ class HackCache:
                  dtype: int, head_is_contextual, budget_c: int, budget_s: int, n_obs: int = 32,
                  n_init_scales: int = 2, sm_scale: float = 0.0,
                  overflow_policy: int = HACK_OVERFLOW_KEEP_PROTECTED, device: int = 0,
-                 obs_sampler: int = HACK_OBS_UNIFORM):
+                 obs_sampler: int = HACK_OBS_UNIFORM, merge_last: bool = False):
         self._h = C.c_void_p()
         sides_arr = (C.c_int32 * len(sides))(*[int(s) for s in sides])
         flat = [int(v) for v in (head_is_contextual.reshape(-1).tolist()
@@ -157,7 +158,7 @@ class HackCache:
             raise ValueError("head_is_contextual must have n_layers*n_heads entries")
         cfg = HackConfig(n_layers, n_heads, head_dim, batch, len(sides), sides_arr, dtype, mask_arr,
                          budget_c, budget_s, n_obs, n_init_scales, sm_scale, overflow_policy, device,
-                         obs_sampler)
+                         obs_sampler, 1 if merge_last else 0)
         _check(lib.hack_init_cache(C.byref(cfg), C.byref(self._h)))
         self.n_layers, self.n_heads, self.head_dim, self.batch = n_layers, n_heads, head_dim, batch
         self.dtype = dtype

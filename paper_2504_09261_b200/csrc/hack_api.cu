@@ -75,6 +75,8 @@ struct hack_cache {
   hack::Scratch scratch{};
   int* status = nullptr;
   int32_t* n_old = nullptr;                     // [b*H] scratch of the compaction kernels
+  hack::MergeScratch merge{};                   // merge_last: scratch of the final-scale merge
+  TensorMapBox merge_ev_map;
   float* attn_row_stats = nullptr;              // bf16 caches: [b*H, max N_k, 2] softmax row statistics (Eq. 6 path)
   float* attn_block_var = nullptr;              // bf16 caches: [b*H, var_blocks] per key block variances
   int var_blocks = 0;
@@ -282,6 +284,8 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
   if (cfg->dtype != HACK_F32 && cfg->dtype != HACK_BF16) return fail(HACK_ERR_UNSUPPORTED, "dtype must be HACK_F32 or HACK_BF16");
   if (cfg->n_obs < 1 || cfg->n_obs > hack::kMaxObs) return fail(HACK_ERR_UNSUPPORTED, "n_obs must be in 1..32");
   if (cfg->obs_sampler < HACK_OBS_UNIFORM || cfg->obs_sampler > HACK_OBS_CALLER) return fail(HACK_ERR_INVALID_ARG, "unknown obs_sampler");
+  if (cfg->merge_last != 0 && cfg->merge_last != 1) return fail(HACK_ERR_INVALID_ARG, "merge_last must be 0 or 1");
+  if (cfg->merge_last && cfg->dtype != HACK_BF16) return fail(HACK_ERR_UNSUPPORTED, "merge_last needs a bf16 cache");
   for (int k = 0; k < cfg->n_scales; ++k)
     if (cfg->scale_sides[k] < 1 || cfg->scale_sides[k] > 1024) return fail(HACK_ERR_INVALID_ARG, "scale side out of range (1..1024)");
   for (int i = 0; i < cfg->n_layers * cfg->n_heads; ++i)
@@ -409,6 +413,32 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
     HACK_TRY(cudaMalloc(&c->attn_row_stats, (size_t)bh * c->limits.max_new * 2 * sizeof(float)));
     HACK_TRY(cudaMalloc(&c->attn_block_var, (size_t)bh * c->var_blocks * sizeof(float)));
   }
+  if (cfg->merge_last) {
+    // what the contextual heads discard at the last scale
+    LayerState ls;
+    hack_step_info_t p{};
+    for (int k = 0; k < cfg->n_scales; ++k) {
+      plan_step(c, ls, k, &p);
+      ls.len[0] = p.kept_s;
+      ls.len[1] = p.kept_c;
+    }
+    hack::MergeScratch& m = c->merge;
+    m.stride = ((std::max(p.cand_c - p.kept_c, 1) + 127) / 128) * 128;
+    const size_t rows = (size_t)bh * m.stride;
+    HACK_TRY(cudaMalloc(&m.ev_k, rows * row_bytes));
+    HACK_TRY(cudaMalloc(&m.ev_v, rows * row_bytes));
+    HACK_TRY(cudaMemset(m.ev_k, 0, rows * row_bytes));
+    HACK_TRY(cudaMalloc(&m.ev_idx, rows * sizeof(int32_t)));
+    HACK_TRY(cudaMalloc(&m.ev_inv_norm, rows * sizeof(float)));
+    HACK_TRY(cudaMalloc(&m.kept_inv_norm, (size_t)bh * c->limits.kept_stride * sizeof(float)));
+    HACK_TRY(cudaMalloc(&m.assign, rows * sizeof(int32_t)));
+    HACK_TRY(cudaMalloc(&m.weight, rows * sizeof(float)));
+    if (!hack::make_rows_map(&c->merge_ev_map, m.ev_k, rows, cfg->head_dim)) {
+      set_error("cuTensorMapEncodeTiled failed for the merge scratch");
+      return bail(HACK_ERR_CUDA);
+    }
+    m.ev_map = &c->merge_ev_map;
+  }
   if (cfg->obs_sampler == HACK_OBS_CALLER) {
     HACK_TRY(cudaMalloc(&c->obs_rows, (size_t)cfg->n_scales * hack::kMaxObs * sizeof(int32_t)));
     HACK_TRY(cudaMemset(c->obs_rows, 0, (size_t)cfg->n_scales * hack::kMaxObs * sizeof(int32_t)));
@@ -431,6 +461,13 @@ hack_status_t hack_free_cache(hack_cache_t* c) {
   cudaFree(c->scratch.logits); cudaFree(c->scratch.partials); cudaFree(c->status);
   cudaFree(c->head_order);
   cudaFree(c->n_old);
+  cudaFree(c->merge.ev_k);
+  cudaFree(c->merge.ev_v);
+  cudaFree(c->merge.ev_idx);
+  cudaFree(c->merge.ev_inv_norm);
+  cudaFree(c->merge.kept_inv_norm);
+  cudaFree(c->merge.assign);
+  cudaFree(c->merge.weight);
   cudaFree(c->attn_row_stats);
   cudaFree(c->attn_block_var);
   cudaFree(c->obs_rows);
@@ -523,6 +560,25 @@ hack_status_t hack_select(hack_cache_t* c, int32_t layer, int32_t scale, const f
   return HACK_OK;
 }
 
+// Compaction of one step; with merge_last, at the last scale, wrapped in the merge of what the
+// contextual heads discard.  Returns the number of launches, or -1.
+static int compact_stage(hack_cache* c, const hack::StepArgs& a, const hack_step_info_t& p, int scale,
+                         const int32_t* idx, int idx_all, const void* k_new, const void* v_new, cudaStream_t st) {
+  const bool merge = c->cfg.merge_last && scale == c->cfg.n_scales - 1 && p.triggered_c && idx;
+  int n = 0, r;
+  if (merge) {
+    if ((r = hack::launch_merge_prepare(a, c->merge, idx, k_new, v_new, st)) < 0) return -1;
+    n += r;
+  }
+  if ((r = hack::launch_compact(a, c->cfg.dtype, idx, idx_all, k_new, v_new, st)) < 0) return -1;
+  n += r;
+  if (merge) {
+    if ((r = hack::launch_merge_finish(a, c->merge, st)) < 0) return -1;
+    n += r;
+  }
+  return n;
+}
+
 hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const int32_t* idx,
                            const void* k_new, const void* v_new, void* stream) {
   hack_status_t s = check_step(c, layer, scale, 0);
@@ -533,7 +589,7 @@ hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const 
   plan_step(c, c->layers[layer], scale, &p);
   const hack::StepArgs a = make_args(c, layer, scale, p);
   StageScope ts(c, (cudaStream_t)stream, 2);
-  const int n = hack::launch_compact(a, c->cfg.dtype, idx, 1, k_new, v_new, (cudaStream_t)stream);
+  const int n = compact_stage(c, a, p, scale, idx, 1, k_new, v_new, (cudaStream_t)stream);
   if (n < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
   ts.done(n);
   c->launches += n;
@@ -649,7 +705,7 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
   }
   {
     StageScope ts(c, st, 2);
-    if ((r = hack::launch_compact(a, c->cfg.dtype, any ? c->idx : nullptr, any ? 1 : 0, k, v, st)) < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
+    if ((r = compact_stage(c, a, p, scale, any ? c->idx : nullptr, any ? 1 : 0, k, v, st)) < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
     ts.done(r);
     n += r;
   }

@@ -51,6 +51,24 @@ struct Scratch {
   int max_chunks;
 };
 
+// Scratch of the final-scale merge of contextual heads (bf16 caches): the rows the last step
+// discards, their list, inverse key norms, and the counterpart and weight of every discarded row.
+struct MergeScratch {
+  int stride;                  // rows per (batch, head) in the arrays below
+  __nv_bfloat16* ev_k;         // [b*H, stride, D] discarded key rows
+  __nv_bfloat16* ev_v;         // [b*H, stride, D] discarded value rows
+  int32_t* ev_idx;             // [b*H, stride] their candidate indices, ascending
+  float* ev_inv_norm;          // [b*H, stride] 1 / |k_e|
+  float* kept_inv_norm;        // [b*H, kept_stride] 1 / |k_c|
+  int32_t* assign;             // [b*H, stride] retained row each discarded row is folded into
+  float* weight;               // [b*H, stride] max(cosine similarity, 0)
+  const void* ev_map;          // host pointer to the 128-byte tensor map over ev_k
+};
+// Before the compaction of the step (idx = the kept lists of launch_select) and after it.
+int launch_merge_prepare(const StepArgs& a, const MergeScratch& ms, const int32_t* idx, const void* k_new,
+                         const void* v_new, cudaStream_t st);
+int launch_merge_finish(const StepArgs& a, const MergeScratch& ms, cudaStream_t st);
+
 // Kernel launchers (each returns the number of kernels it enqueued, or -1 on a launch error).
 int launch_score(const StepArgs& a, int dtype, const void* q, const void* k_new, float* scores,
                  const Scratch& s, cudaStream_t st);

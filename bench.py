@@ -33,7 +33,7 @@ METRIC = "scale-step tokens/s (score+select+compact+attend)"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one last-scale attention launch, from the ncu
 # capture summarised in profiles/attend_tc_config3_last_scale.md (same launch shape as the bench's)
-ATTEND_LAST_SCALE_DRAM_BYTES = {3: 85371136 + 8060928}
+ATTEND_LAST_SCALE_DRAM_BYTES = {3: 85393408 + 11214848}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

@@ -37,6 +37,7 @@ constexpr int kRing = 2;
 constexpr int kApplyThreads = 256;
 constexpr int kApplyRowsPerWarp = 8;     // retained rows per warp (64 per CTA)
 constexpr int kApplyChunk = 2048;        // discarded entries staged in shared memory at a time
+constexpr int kApplyHits = 256;          // entries a warp lists before it works them off
 constexpr long long kMergeWaitCycles = 2000000000ll;   // about one second
 constexpr uint32_t kMergeDrainSpins = 1u << 22;
 
@@ -322,8 +323,9 @@ merge_assign_kernel(const __grid_constant__ CUtensorMap tm_e, const __grid_const
 
 // ---------------------------------------------------------------- weighted average into the retained rows
 // A warp owns kApplyRowsPerWarp consecutive retained rows and walks the list of discarded entries
-// once; an entry assigned to one of its rows is added to that row's fp32 accumulator in shared
-// memory.  Entries are taken in ascending order, so a row's sum has one fixed order of additions.
+// once, listing those assigned to its rows; the listed rows are then fetched eight at a time and
+// added to the rows' fp32 accumulators in shared memory.  Entries are taken in ascending order,
+// so a row's sum has one fixed order of additions.
 template <int D>
 __global__ void __launch_bounds__(kApplyThreads)
 merge_apply_kernel(const StepArgs a, const MergeScratch ms) {
@@ -340,82 +342,88 @@ merge_apply_kernel(const StepArgs a, const MergeScratch ms) {
   float* den_all = acc_all + kWarps * R * 2 * D;                          // [warp][row]
   int* s_assign = reinterpret_cast<int*>(den_all + kWarps * R);           // [kApplyChunk]
   float* s_weight = reinterpret_cast<float*>(s_assign + kApplyChunk);     // [kApplyChunk]
+  int* s_hits = reinterpret_cast<int*>(s_weight + kApplyChunk);           // [warp][kApplyHits]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c0 = (blockIdx.x * kWarps + warp) * R;
   float* acc = acc_all + warp * R * 2 * D;
   float* den = den_all + warp * R;
   for (int i = lane; i < R * 2 * D; i += 32) acc[i] = 0.f;
   if (lane < R) den[lane] = 0.f;
+  int* hits = s_hits + warp * kApplyHits;                       // entries of this chunk assigned to this warp's rows
+  // adds up to 8 listed entries: their rows are fetched together (the latencies overlap), then added in order
+  auto flush = [&](int base, int n_hits) {
+    for (int h0 = 0; h0 < n_hits; h0 += 8) {
+      Vec kv[8], vv[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (h0 + u < n_hits) {
+          const size_t row = ((size_t)bh * ms.stride + base + hits[h0 + u]) * D;
+          kv[u] = reinterpret_cast<const Vec*>(ms.ev_k + row)[lane];
+          vv[u] = reinterpret_cast<const Vec*>(ms.ev_v + row)[lane];
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (h0 + u < n_hits) {
+          const int el = hits[h0 + u];
+          const int r = s_assign[el] - c0;
+          const float w = s_weight[el];
+          const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(&kv[u]);
+          const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vv[u]);
+          float* ak = acc + (r * 2) * D + lane * E;
+          float* av = ak + D;
+#pragma unroll
+          for (int x = 0; x < E; ++x) {
+            ak[x] = fmaf(w, __bfloat162float(ke[x]), ak[x]);
+            av[x] = fmaf(w, __bfloat162float(ve[x]), av[x]);
+          }
+          if (lane == 0) den[r] += w;
+        }
+      }
+    }
+    __syncwarp();
+  };
   for (int base = 0; base < n_evict; base += kApplyChunk) {
     const int n = min(kApplyChunk, n_evict - base);
+    const int n_pad = (n + 127) & ~127;
     __syncthreads();
-    for (int i = threadIdx.x; i < ((n + 127) & ~127); i += kApplyThreads) {
+#pragma unroll 4
+    for (int i = threadIdx.x; i < n_pad; i += kApplyThreads) {
       s_assign[i] = i < n ? ms.assign[(size_t)bh * ms.stride + base + i] : -1;
       s_weight[i] = i < n ? ms.weight[(size_t)bh * ms.stride + base + i] : 0.f;
     }
     __syncthreads();
     if (c0 >= kept) continue;
     // 128 entries per pass: a lane looks at four consecutive ones (entries past the chunk's end
-    // were staged as -1); an entry with weight 0 adds nothing and needs no test here
+    // were staged as -1); an entry with weight 0 adds nothing and needs no test here.  Hits go to
+    // the warp's list in ascending order; the list is worked off when it fills and at the end.
+    int n_hits = 0;
     for (int e4 = 0; e4 < n; e4 += 128) {
       const int4 as = *reinterpret_cast<const int4*>(&s_assign[e4 + lane * 4]);
-      const bool h0 = (unsigned)(as.x - c0) < (unsigned)R, h1 = (unsigned)(as.y - c0) < (unsigned)R;
-      const bool h2 = (unsigned)(as.z - c0) < (unsigned)R, h3 = (unsigned)(as.w - c0) < (unsigned)R;
-      if (!__any_sync(0xffffffffu, h0 | h1 | h2 | h3)) continue;
-      // bit 4 * lane + j of the 128-bit hit mask, walked in ascending entry order 32 bits at a time
-      const uint32_t mine = (h0 ? 1u : 0u) | (h1 ? 2u : 0u) | (h2 ? 4u : 0u) | (h3 ? 8u : 0u);
-#pragma unroll 1
-      for (int part = 0; part < 4; ++part) {
-      const uint32_t nib = __shfl_sync(0xffffffffu, mine, part * 8 + (lane >> 2));
-      uint32_t m = __ballot_sync(0xffffffffu, (nib >> (lane & 3)) & 1u);
-      const int e0 = e4 + part * 32;
-      auto add_row = [&](int el, const Vec& kv, const Vec& vv) {
-        const int r = s_assign[el] - c0;
-        const float w = s_weight[el];
-        const __nv_bfloat16* ke = reinterpret_cast<const __nv_bfloat16*>(&kv);
-        const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vv);
-        float* ak = acc + (r * 2) * D + lane * E;
-        float* av = ak + D;
-#pragma unroll
-        for (int x = 0; x < E; ++x) {
-          ak[x] = fmaf(w, __bfloat162float(ke[x]), ak[x]);
-          av[x] = fmaf(w, __bfloat162float(ve[x]), av[x]);
-        }
-        if (lane == 0) den[r] += w;
-      };
-      if (m && (m & (m - 1)) == 0) {                            // the usual case: one entry among these 32
-        const int el = e0 + __ffs(m) - 1;
-        const size_t row = ((size_t)bh * ms.stride + base + el) * D;
-        add_row(el, reinterpret_cast<const Vec*>(ms.ev_k + row)[lane], reinterpret_cast<const Vec*>(ms.ev_v + row)[lane]);
-        m = 0;
+      const uint32_t mine = ((unsigned)(as.x - c0) < (unsigned)R ? 1u : 0u) | ((unsigned)(as.y - c0) < (unsigned)R ? 2u : 0u) |
+                            ((unsigned)(as.z - c0) < (unsigned)R ? 4u : 0u) | ((unsigned)(as.w - c0) < (unsigned)R ? 8u : 0u);
+      if (!__any_sync(0xffffffffu, mine != 0u)) continue;
+      if (n_hits + 128 > kApplyHits) {
+        __syncwarp();
+        flush(base, n_hits);
+        n_hits = 0;
       }
-      while (m) {
-        // up to kBatch rows are fetched together (their latencies overlap) and added in order
-        constexpr int kBatch = 4;
-        int el[kBatch];
-        Vec kv[kBatch], vv[kBatch];
+      // position of this lane's hits = hits of the lower lanes (ascending entry order)
+      const int cnt = __popc(mine);
+      int incl = cnt;
 #pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-          el[u] = -1;
-          if (m) {
-            el[u] = e0 + __ffs(m) - 1;
-            m &= m - 1;
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-          if (el[u] >= 0) {
-            const size_t row = ((size_t)bh * ms.stride + base + el[u]) * D;
-            kv[u] = reinterpret_cast<const Vec*>(ms.ev_k + row)[lane];
-            vv[u] = reinterpret_cast<const Vec*>(ms.ev_v + row)[lane];
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u)
-          if (el[u] >= 0) add_row(el[u], kv[u], vv[u]);
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
       }
-      }
+      int pos = n_hits + incl - cnt;
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (mine & (1u << j)) hits[pos++] = e4 + lane * 4 + j;
+      n_hits += __shfl_sync(0xffffffffu, incl, 31);
     }
+    __syncwarp();
+    flush(base, n_hits);
   }
   __syncwarp();
   for (int r = 0; r < R; ++r) {
@@ -444,7 +452,7 @@ merge_apply_kernel(const StepArgs a, const MergeScratch ms) {
 
 template <int D>
 size_t apply_smem_bytes() {
-  return ((size_t)(kApplyThreads / 32) * kApplyRowsPerWarp * (2 * D + 1) + 2 * kApplyChunk) * sizeof(float);
+  return ((size_t)(kApplyThreads / 32) * (kApplyRowsPerWarp * (2 * D + 1) + kApplyHits) + 2 * kApplyChunk) * sizeof(float);
 }
 
 template <int D>

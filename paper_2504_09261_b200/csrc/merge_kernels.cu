@@ -323,11 +323,11 @@ merge_assign_kernel(const __grid_constant__ CUtensorMap tm_e, const __grid_const
 
 // ---------------------------------------------------------------- weighted average into the retained rows
 // A warp owns kApplyRowsPerWarp consecutive retained rows and walks the list of discarded entries
-// once, listing those assigned to its rows; the listed rows are then fetched eight at a time and
+// once, listing those assigned to its rows; the listed rows are then fetched four at a time and
 // added to the rows' fp32 accumulators in shared memory.  Entries are taken in ascending order,
 // so a row's sum has one fixed order of additions.
 template <int D>
-__global__ void __launch_bounds__(kApplyThreads)
+__global__ void __launch_bounds__(kApplyThreads, 2)
 merge_apply_kernel(const StepArgs a, const MergeScratch ms) {
   pdl_wait();
   const int bh = blockIdx.y;
@@ -350,12 +350,12 @@ merge_apply_kernel(const StepArgs a, const MergeScratch ms) {
   for (int i = lane; i < R * 2 * D; i += 32) acc[i] = 0.f;
   if (lane < R) den[lane] = 0.f;
   int* hits = s_hits + warp * kApplyHits;                       // entries of this chunk assigned to this warp's rows
-  // adds up to 8 listed entries: their rows are fetched together (the latencies overlap), then added in order
+  // adds the listed entries, four at a time: their rows are fetched together (the latencies overlap), then added in order
   auto flush = [&](int base, int n_hits) {
-    for (int h0 = 0; h0 < n_hits; h0 += 8) {
-      Vec kv[8], vv[8];
+    for (int h0 = 0; h0 < n_hits; h0 += 4) {
+      Vec kv[4], vv[4];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
+      for (int u = 0; u < 4; ++u) {
         if (h0 + u < n_hits) {
           const size_t row = ((size_t)bh * ms.stride + base + hits[h0 + u]) * D;
           kv[u] = reinterpret_cast<const Vec*>(ms.ev_k + row)[lane];
@@ -363,7 +363,7 @@ merge_apply_kernel(const StepArgs a, const MergeScratch ms) {
         }
       }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
+      for (int u = 0; u < 4; ++u) {
         if (h0 + u < n_hits) {
           const int el = hits[h0 + u];
           const int r = s_assign[el] - c0;
@@ -426,27 +426,33 @@ merge_apply_kernel(const StepArgs a, const MergeScratch ms) {
     flush(base, n_hits);
   }
   __syncwarp();
-  for (int r = 0; r < R; ++r) {
-    const int c = c0 + r;
-    if (c >= kept) break;
-    const float d = den[r];
-    if (d == 0.f) continue;                                    // nothing was assigned: the row keeps its bits
-    const float inv = 1.f / (1.f + d);
-    __nv_bfloat16* kr = static_cast<__nv_bfloat16*>(a.k_plane) + ((size_t)a.row_off[bh] + c) * D;
-    __nv_bfloat16* vr = static_cast<__nv_bfloat16*>(a.v_plane) + ((size_t)a.row_off[bh] + c) * D;
-    Vec kv = reinterpret_cast<const Vec*>(kr)[lane];
-    Vec vv = reinterpret_cast<const Vec*>(vr)[lane];
-    __nv_bfloat16* ke = reinterpret_cast<__nv_bfloat16*>(&kv);
-    __nv_bfloat16* ve = reinterpret_cast<__nv_bfloat16*>(&vv);
-    const float* ak = acc + (r * 2) * D + lane * E;
-    const float* av = ak + D;
+  // the rows that received something: all of them are fetched before any is written back
+  Vec kv[R], vv[R];
 #pragma unroll
-    for (int x = 0; x < E; ++x) {
-      ke[x] = __float2bfloat16_rn((__bfloat162float(ke[x]) + ak[x]) * inv);
-      ve[x] = __float2bfloat16_rn((__bfloat162float(ve[x]) + av[x]) * inv);
+  for (int r = 0; r < R; ++r) {
+    if (c0 + r < kept && den[r] != 0.f) {
+      const size_t row = ((size_t)a.row_off[bh] + c0 + r) * D;
+      kv[r] = reinterpret_cast<const Vec*>(static_cast<const __nv_bfloat16*>(a.k_plane) + row)[lane];
+      vv[r] = reinterpret_cast<const Vec*>(static_cast<const __nv_bfloat16*>(a.v_plane) + row)[lane];
     }
-    reinterpret_cast<Vec*>(kr)[lane] = kv;
-    reinterpret_cast<Vec*>(vr)[lane] = vv;
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    if (c0 + r < kept && den[r] != 0.f) {                      // else nothing was assigned: the row keeps its bits
+      const float inv = 1.f / (1.f + den[r]);
+      __nv_bfloat16* ke = reinterpret_cast<__nv_bfloat16*>(&kv[r]);
+      __nv_bfloat16* ve = reinterpret_cast<__nv_bfloat16*>(&vv[r]);
+      const float* ak = acc + (r * 2) * D + lane * E;
+      const float* av = ak + D;
+#pragma unroll
+      for (int x = 0; x < E; ++x) {
+        ke[x] = __float2bfloat16_rn((__bfloat162float(ke[x]) + ak[x]) * inv);
+        ve[x] = __float2bfloat16_rn((__bfloat162float(ve[x]) + av[x]) * inv);
+      }
+      const size_t row = ((size_t)a.row_off[bh] + c0 + r) * D;
+      reinterpret_cast<Vec*>(static_cast<__nv_bfloat16*>(a.k_plane) + row)[lane] = kv[r];
+      reinterpret_cast<Vec*>(static_cast<__nv_bfloat16*>(a.v_plane) + row)[lane] = vv[r];
+    }
   }
 }
 

@@ -202,6 +202,9 @@ def run_ours(args):
     cfg = get_config(args.config)
     if args.layers:
         cfg = cfg.with_layers(args.layers)
+    if args.n_obs:
+        from dataclasses import replace as _replace
+        cfg = _replace(cfg, n_obs=args.n_obs)
     L, K = cfg.n_layers, cfg.n_scales
     gen = sharding.rank_generator(cfg, rank, device=dev)        # each rank decodes its own images
     mask = gen.head_is_contextual
@@ -211,7 +214,7 @@ def run_ours(args):
     def new_cache(bc, bs, policy=0):
         return hb.HackCache(L, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides, dtype_id, mask.numpy(),
                             bc, bs, n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, overflow_policy=policy,
-                            device=local, merge_last=args.merge_last)
+                            device=local, merge_last=args.merge_last, obs_sampler=args.obs_sampler)
 
     cache = new_cache(cfg.budget_c, cfg.budget_s)
     # inputs resident in HBM: every (layer, scale) has its own Q, K, V (ranks draw different images)
@@ -631,6 +634,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--n-obs", type=int, default=0, help="query subset size N_obs (1..32) instead of the workload's 32")
+    ap.add_argument("--obs-sampler", type=int, default=0, choices=[0, 1, 2],
+                    help="query subset rule: 0 uniform (the method), 1 first n, 2 last n")
     ap.add_argument("--merge-last", action="store_true",
                     help="contextual heads fold what the last scale discards into what it keeps (off in the paper's efficiency runs' default here)")
     ap.add_argument("--latency-profile", action="store_true",

@@ -67,8 +67,10 @@ enum { HACK_OVERFLOW_KEEP_PROTECTED = 0, /* keep every protected entry, exceed B
 enum { HACK_OBS_UNIFORM = 0, /* floor(m * N_k / n), m = 0..n-1 */
        HACK_OBS_INIT = 1,    /* the first n tokens of the scale */
        HACK_OBS_RECENT = 2,  /* the last n tokens of the scale */
-       HACK_OBS_CALLER = 3 };/* rows given per scale with hack_set_obs_rows (random sampling: the
+       HACK_OBS_CALLER = 3,  /* rows given per scale with hack_set_obs_rows (random sampling: the
                                 caller draws them) */
+       HACK_OBS_FULL = 4 };  /* every query of the scale, whatever n_obs: the ablation's full-attention
+                                reference; costs ceil(N_k / 32) scoring rounds per step */
 
 typedef struct {
   int32_t n_layers, n_heads, head_dim, batch; /* head_dim in {64, 128} */

@@ -58,7 +58,7 @@ def split_budget(budget: int, alpha: float, rule: str, param: float, total_token
 
 
 # --------------------------------------------------------------------------- step pieces
-UNIFORM, INIT, RECENT, CALLER = 0, 1, 2, 3   # query-subset rules of the sampling ablation (Table "qselect")
+UNIFORM, INIT, RECENT, CALLER, FULL = 0, 1, 2, 3, 4   # query-subset rules of the sampling ablation
 
 
 def observation_rows(n_k: int, n_obs: int, sampler: int = UNIFORM,
@@ -67,8 +67,11 @@ def observation_rows(n_k: int, n_obs: int, sampler: int = UNIFORM,
 
     UNIFORM (the method's rule): floor(m * N_k / n).  INIT: the first n tokens.  RECENT: the last n
     tokens.  CALLER: rows drawn outside (the ablation's random sampling), n distinct indices given in
-    `caller_rows`, used in the order given.  The last three are the alternatives the paper's
-    query-subset ablation compares the uniform rule with."""
+    `caller_rows`, used in the order given.  FULL: every query of the scale, whatever N_obs (the
+    ablation's "full attention" reference).  These are the alternatives the paper's query-subset
+    ablation compares the uniform rule with."""
+    if sampler == FULL:
+        return np.arange(n_k, dtype=np.int64)
     n = min(n_obs, n_k)
     if sampler == UNIFORM:
         return np.array([(m * n_k) // n for m in range(n)], dtype=np.int64)

@@ -16,7 +16,7 @@ HACK_OK, HACK_ERR_INVALID_ARG, HACK_ERR_UNSUPPORTED, HACK_ERR_OOM, HACK_ERR_CUDA
     HACK_ERR_TIMEOUT = range(7)
 HACK_F32, HACK_BF16 = 0, 1
 HACK_OVERFLOW_KEEP_PROTECTED, HACK_OVERFLOW_COMPETE = 0, 1
-HACK_OBS_UNIFORM, HACK_OBS_INIT, HACK_OBS_RECENT, HACK_OBS_CALLER = 0, 1, 2, 3
+HACK_OBS_UNIFORM, HACK_OBS_INIT, HACK_OBS_RECENT, HACK_OBS_CALLER, HACK_OBS_FULL = 0, 1, 2, 3, 4
 RULE_FRACTION, RULE_RATIO = 0, 1
 
 EXPORTS = (

@@ -164,6 +164,7 @@ hack::StepArgs make_args(const hack_cache* c, int layer, int scale, const hack_s
   a.obs_first = c->cfg.obs_sampler == HACK_OBS_RECENT ? p.n_new - p.n_obs_rows : 0;
   a.obs_span = c->cfg.obs_sampler == HACK_OBS_UNIFORM ? p.n_new : p.n_obs_rows;
   a.obs_rows = c->cfg.obs_sampler == HACK_OBS_CALLER ? c->obs_rows + (size_t)scale * hack::kMaxObs : nullptr;
+  a.obs_full = c->cfg.obs_sampler == HACK_OBS_FULL;
   a.sm_scale = c->sm_scale;
   a.t_init = c->t_init;
   a.protect_new = (c->cfg.overflow_policy == HACK_OVERFLOW_KEEP_PROTECTED) || scale < c->cfg.n_init_scales;
@@ -283,7 +284,7 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return fail(HACK_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
   if (cfg->dtype != HACK_F32 && cfg->dtype != HACK_BF16) return fail(HACK_ERR_UNSUPPORTED, "dtype must be HACK_F32 or HACK_BF16");
   if (cfg->n_obs < 1 || cfg->n_obs > hack::kMaxObs) return fail(HACK_ERR_UNSUPPORTED, "n_obs must be in 1..32");
-  if (cfg->obs_sampler < HACK_OBS_UNIFORM || cfg->obs_sampler > HACK_OBS_CALLER) return fail(HACK_ERR_INVALID_ARG, "unknown obs_sampler");
+  if (cfg->obs_sampler < HACK_OBS_UNIFORM || cfg->obs_sampler > HACK_OBS_FULL) return fail(HACK_ERR_INVALID_ARG, "unknown obs_sampler");
   if (cfg->merge_last != 0 && cfg->merge_last != 1) return fail(HACK_ERR_INVALID_ARG, "merge_last must be 0 or 1");
   if (cfg->merge_last && cfg->dtype != HACK_BF16) return fail(HACK_ERR_UNSUPPORTED, "merge_last needs a bf16 cache");
   for (int k = 0; k < cfg->n_scales; ++k)

@@ -27,6 +27,8 @@ struct StepArgs {
   int n_obs_rows;       // min(N_obs, N_k)
   int obs_first, obs_span;      // observation row i = obs_first + floor(i * obs_span / n_obs_rows) ...
   const int32_t* obs_rows;      // ... unless the caller supplied the rows (device, [n_obs_rows])
+  int obs_full;                 // every query observes: the scoring kernels run once per group of 32 rows
+  int score_accumulate;         // the scores of this round are added to those already there
   float sm_scale;
   int t_init;           // tokens in the always-kept leading scales (structural heads)
   int protect_new;      // structural heads: the new scale's tokens are protected

@@ -5,6 +5,8 @@
 // the (at most 32) observation rows, stores them to scratch and publishes per-row (max, sum-exp)
 // partials for its chunk.  Pass 2 merges the partials into the row statistics of the full
 // softmax over all T' candidates and reduces every column: s_j = sum_i exp(z_ij - m_i) / l_i.
+#include <algorithm>
+
 #include "hack_internal.h"
 
 namespace hack {
@@ -168,7 +170,8 @@ score_reduce_kernel(const StepArgs a, const float* __restrict__ logits,
     const float z = logits[((size_t)bh * kMaxObs + i) * a.cand_stride + j];
     s += expf(z - row_m[i]) * row_inv_l[i];
   }
-  scores[(size_t)bh * a.cand_stride + j] = s;
+  float* dst = scores + (size_t)bh * a.cand_stride + j;
+  *dst = a.score_accumulate ? *dst + s : s;
 }
 
 template <typename T, int D>
@@ -190,9 +193,8 @@ int launch_score_t(const StepArgs& a, const void* q, const void* k_new, float* s
 
 }  // namespace
 
-int launch_score(const StepArgs& a, int dtype, const void* q, const void* k_new, float* scores,
-                 const Scratch& s, cudaStream_t st) {
-  if (!a.trig[0] && !a.trig[1]) return 0;
+static int launch_score_round(const StepArgs& a, int dtype, const void* q, const void* k_new, float* scores,
+                              const Scratch& s, cudaStream_t st) {
   // bf16: tensor-core kernel, unless the new K tensor has fewer rows than one TMA box
   if (dtype == HACK_BF16 && a.k_map && (long long)a.batch * a.n_heads * a.n_new >= 128)
     return launch_score_tc(a, q, k_new, scores, s, st);
@@ -202,6 +204,27 @@ int launch_score(const StepArgs& a, int dtype, const void* q, const void* k_new,
   }
   return a.head_dim == 64 ? launch_score_t<__nv_bfloat16, 64>(a, q, k_new, scores, s, st)
                           : launch_score_t<__nv_bfloat16, 128>(a, q, k_new, scores, s, st);
+}
+
+int launch_score(const StepArgs& a, int dtype, const void* q, const void* k_new, float* scores,
+                 const Scratch& s, cudaStream_t st) {
+  if (!a.trig[0] && !a.trig[1]) return 0;
+  if (!a.obs_full) return launch_score_round(a, dtype, q, k_new, scores, s, st);
+  // every query observes: one scoring round per group of kMaxObs consecutive query rows; every
+  // row's softmax is normalised over all candidates inside its round, so the rounds simply add up
+  int n = 0;
+  for (int first = 0; first < a.n_new; first += kMaxObs) {
+    StepArgs g = a;
+    g.n_obs_rows = std::min(kMaxObs, a.n_new - first);
+    g.obs_first = first;
+    g.obs_span = g.n_obs_rows;
+    g.obs_rows = nullptr;
+    g.score_accumulate = first > 0;
+    const int r = launch_score_round(g, dtype, q, k_new, scores, s, st);
+    if (r < 0) return r;
+    n += r;
+  }
+  return n;
 }
 
 }  // namespace hack

@@ -260,7 +260,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_const
         float s = 0.f;
 #pragma unroll
         for (int r = 0; r < kMaxObs; ++r) s = fmaf(ex2(fmaf(__uint_as_float(acc[r]), zscale, -rm[r])), rl[r], s);
-        if (live) scores[(size_t)bh * a.cand_stride + (from_cache ? 0 : stored) + part_row + key_row] = s;
+        if (live) {
+          float* dst = scores + (size_t)bh * a.cand_stride + (from_cache ? 0 : stored) + part_row + key_row;
+          *dst = a.score_accumulate ? *dst + s : s;
+        }
       }
     }
     if (MODE == 1 && ok) {

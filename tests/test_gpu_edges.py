@@ -69,15 +69,16 @@ def test_single_observation_row_and_single_scale():
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("sampler", ["init", "recent", "caller"])
+@pytest.mark.parametrize("sampler", ["init", "recent", "caller", "full"])
 def test_query_subset_rules_of_the_ablation(sampler, dtype):
     """The alternatives the paper's query-subset ablation compares with uniform spacing (first n,
-    last n, random rows drawn by the caller) against the oracle under the same rule, with N_obs = 8
+    last n, random rows drawn by the caller, and every query: the ablation's reference) against the oracle under the same rule, with N_obs = 8
     and 32 so that both subset sizes of the size ablation's range and a ragged last scale occur."""
     import paper_2504_09261_b200 as hb
     from workloads import random_observation_rows
     from tests.parity_util import run_parity
-    code = {"init": hb.HACK_OBS_INIT, "recent": hb.HACK_OBS_RECENT, "caller": hb.HACK_OBS_CALLER}[sampler]
+    code = {"init": hb.HACK_OBS_INIT, "recent": hb.HACK_OBS_RECENT, "caller": hb.HACK_OBS_CALLER,
+            "full": hb.HACK_OBS_FULL}[sampler]
     for n_obs in (8, 32):
         cfg = _custom(1 if dtype == "bf16" else 0, n_obs=n_obs, n_heads=4, batch=1, dtype=dtype,
                       sides=(1, 2, 3, 5, 8, 13, 19))

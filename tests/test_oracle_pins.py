@@ -111,6 +111,25 @@ def test_observation_rows_of_the_ablation_samplers():
     for bad in ([0, 1, 2], [0, 1, 2, 2], [0, 1, 2, 10], [-1, 1, 2, 3]):
         with pytest.raises(ValueError):
             ho.observation_rows(10, 4, ho.CALLER, bad)
+    assert list(ho.observation_rows(10, 4, ho.FULL)) == list(range(10))
+
+
+def test_full_query_set_scores_are_the_column_sums_of_the_attention_matrix():
+    """With every query observing, a contextual step keeps the keys with the largest column sums of
+    the step's whole attention matrix (computed here with explicit loops)."""
+    rng = np.random.default_rng(12)
+    D, n_k = 6, 9
+    q, k, v = rng.normal(size=(n_k, D)), rng.normal(size=(n_k, D)), rng.normal(size=(n_k, D))
+    col = [0.0] * n_k
+    for i in range(n_k):
+        z = [sum(q[i, t] * k[j, t] for t in range(D)) / math.sqrt(D) for j in range(n_k)]
+        den = sum(math.exp(x) for x in z)
+        for j in range(n_k):
+            col[j] += math.exp(z[j]) / den
+    orc = ho.HackOracle(1, 1, 1, D, (3,), np.array([[1]]), budget_c=4, budget_s=4, n_obs=2, obs_sampler=ho.FULL)
+    _, rec = orc.head_step(0, 0, 0, 0, q, k, v)
+    np.testing.assert_allclose(rec.scores, col, rtol=1e-12)
+    assert list(rec.keep) == sorted(sorted(range(n_k), key=lambda j: -col[j])[:4])
 
 
 def test_sampler_decides_which_key_a_contextual_head_keeps():

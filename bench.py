@@ -31,10 +31,27 @@ from workloads import sharding  # noqa: E402
 
 METRIC = "scale-step tokens/s (score+select+compact+attend)"
 UNIT = "tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one last-scale attention launch, from the ncu
-# capture summarised in profiles/attend_tc_config3_last_scale.md (same launch shape as the bench's)
-ATTEND_LAST_SCALE_DRAM_BYTES = {3: 85393408 + 11214848}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}      # the figures the target names
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
+
+
+def measured_traffic(config_index: int):
+    """DRAM bytes of one last-scale attention launch as ncu counted them, or None when there is no
+    record for this workload or the kernel source has changed since the counters were taken."""
+    import hashlib
+    try:
+        with open(TRAFFIC_FILE) as f:
+            rec = json.load(f).get(f"attend_tc_config{config_index}_last_scale")
+        if not rec:
+            return None
+        src = os.path.join(ROOT, rec["source"])
+        with open(src, "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != rec["source_sha256"]:
+                return None
+        return int(rec["dram_bytes_read"]) + int(rec["dram_bytes_write"])
+    except Exception:
+        return None
 
 
 def load_peaks():
@@ -199,7 +216,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device(f"cuda:{local}")
 
-    cfg = get_config(args.config)
+    cfg = get_config(args.config, args.budget_frac, args.alpha)
     if args.layers:
         cfg = cfg.with_layers(args.layers)
     if args.n_obs:
@@ -358,7 +375,16 @@ def run_ours(args):
     # ---- work model and roofline of the loop
     peaks, peak_kind = load_peaks()
     hbm = peaks["hbm_gbs"] * 1e9
+    tf_burst = peaks["bf16_tflops"] * 1e12
     tf_sus = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12
+    # Which measured tensor peak is like for like: the burst figure was taken at full clock, the
+    # sustained one under the power cap (about two thirds of the clock).  A run whose sampled SM
+    # clock stayed near the maximum with no power cap is compared with the burst peak.
+    at_full_clock = bool(clocks["sm_mhz"] and clocks["sm_max_mhz"] and clocks["sm_mhz"] >= 0.9 * clocks["sm_max_mhz"]
+                         and "sw_power_cap" not in clocks["reasons"])
+    tf_ref = tf_burst if at_full_clock else tf_sus
+    peak_note = (f"bf16_tflops ({'burst' if at_full_clock else 'sustained'}) of {peak_kind}: median SM clock "
+                 f"{clocks['sm_mhz']} of {clocks['sm_max_mhz']} MHz, reasons {clocks['reasons']}")
     infos = []
     walker = hb.HackCache(1, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides, dtype_id, mask[0].numpy(),
                           cfg.budget_c, cfg.budget_s, n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales,
@@ -373,6 +399,7 @@ def run_ours(args):
     walker.close()
     attend_fl = score_fl = byt = 0.0
     t_roof = 0.0
+    roof_alt = {"sustained": 0.0, "burst": 0.0, "nominal": 0.0}
     per_scale = []
     for k in range(K):
         a_k = s_k = b_k = roof_k = 0.0
@@ -381,7 +408,11 @@ def run_ours(args):
             a_k += a
             s_k += s
             b_k += by
-            roof_k += max((a + s) / tf_sus, by / hbm)
+            roof_k += max((a + s) / tf_ref, by / hbm)
+            roof_alt["sustained"] += max((a + s) / tf_sus, by / hbm)
+            roof_alt["burst"] += max((a + s) / tf_burst, by / hbm)
+            roof_alt["nominal"] += max((a + s) / (NOMINAL_PEAKS["bf16_tflops"] * 1e12),
+                                       by / (NOMINAL_PEAKS["hbm_gbs"] * 1e9))
         attend_fl += a_k
         score_fl += s_k
         byt += b_k
@@ -441,15 +472,17 @@ def run_ours(args):
         last_flops = 4.0 * last.n_new * cfg.head_dim * kept_sum
         last_bytes = 2 * kept_sum * cfg.head_dim * 2 + 2 * last.n_new * bh * cfg.head_dim * 2
         achieved = last_flops / (last_ms * 1e-3) / 1e12
-        peak_tf = tf_sus / 1e12 if cfg.dtype != "f32" else None
+        peak_tf = tf_ref / 1e12 if cfg.dtype != "f32" else None
         att_ms = stage["attend"]["ms_per_step"]
         att_n = max(stage["attend"]["launches_per_step"], 1)
         roofline = {
             "kernel": "attend_tc_kernel, launch of the last scale", "bound": "tensor",
             "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
             "frac": (achieved / peak_tf) if peak_tf else None,
-            "traffic": ATTEND_LAST_SCALE_DRAM_BYTES.get(cfg.index),
-            "peak_source": f"bf16_tflops_sustained of {peak_kind} (the launch runs inside a long step)",
+            "traffic": measured_traffic(cfg.index),
+            "peak_source": peak_note,
+            "frac_of_burst": achieved / (tf_burst / 1e12), "frac_of_sustained": achieved / (tf_sus / 1e12),
+            "frac_of_nominal": achieved / NOMINAL_PEAKS["bf16_tflops"],
             "flops_per_launch": last_flops, "algorithmic_bytes_per_launch": last_bytes,
             "launch_ms_median": last_ms, "launches_timed": len(evs),
             "all_attend_launches": {"tflops": attend_fl / (att_ms * 1e-3) / 1e12, "launches_per_step": att_n,
@@ -503,7 +536,7 @@ def run_ours(args):
     # ---- CPU oracle on the host cores (rank 0, N = 1)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
-        base_cfg = get_config(args.config)
+        base_cfg = get_config(args.config, args.budget_frac, args.alpha)
         dt, frac, threads, used = oracle_sample_run(base_cfg, args.oracle_pairs)
         cpu = {"value": base_cfg.batch * base_cfg.total_tokens / (dt / frac), "unit": UNIT, "cores": threads,
                "kind": "oracle", "seconds_measured": dt,
@@ -527,7 +560,11 @@ def run_ours(args):
             },
             "roofline": roofline,
             "loop_roofline": {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_per_step,
-                              "flops": attend_fl + score_fl, "bytes": byt, "peaks": peak_kind},
+                              "flops": attend_fl + score_fl, "bytes": byt, "peaks": peak_kind,
+                              "tensor_peak": peak_note,
+                              "frac_of_sustained": roof_alt["sustained"] * 1e3 / ms_per_step,
+                              "frac_of_burst": roof_alt["burst"] * 1e3 / ms_per_step,
+                              "frac_of_nominal": roof_alt["nominal"] * 1e3 / ms_per_step},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks, "stages": stage, "per_scale": per_scale,
             "kv_bytes": {"live": live, "peak": peak, "reserved": reserved,
@@ -535,11 +572,13 @@ def run_ours(args):
                          * cfg.n_heads * L * cfg.batch},
             "full_cache_run": full,
         }
-        print(json.dumps(line))
+        if not args.quiet:
+            print(json.dumps(line))
     cache.close()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+    return line if rank == 0 else None
 
 
 def run_head_variance(args):
@@ -621,6 +660,47 @@ def run_head_variance(args):
     cache.close()
 
 
+def run_sweep(args):
+    """Every workload that has budget literals (configs 0, 1, 2 x {30, 50, 70 %}, 3, 4 x {25, 50, 75 %
+    contextual} x {10, 30, 50 %}), one compact JSON line each: loop time, tokens/s, fraction of the
+    loop roofline, KV bytes, and the uncompressed run of the same inputs."""
+    from workloads import list_configs
+    for (index, frac, alpha) in list_configs():
+        a = argparse.Namespace(**vars(args))
+        a.config, a.budget_frac, a.alpha = index, frac, alpha
+        a.no_e2e = a.no_cpu = a.quiet = True
+        a.no_full = False
+        line = run_ours(a)
+        torch.cuda.empty_cache()
+        full = line["full_cache_run"]
+        print(json.dumps({
+            "workload": line["config"]["workload"], "budget_frac": frac, "alpha": alpha,
+            "budget_c": line["config"]["budget_c"], "budget_s": line["config"]["budget_s"],
+            "dtype": line["dtype"], "ms_per_step": round(line["ms_per_step"], 4),
+            "tokens_per_s": round(line["value"], 1), "gpu_launches_per_step": line["gpu_launches"] // line["steps"],
+            "loop_roofline": {k: (round(v, 4) if isinstance(v, float) else v) for k, v in line["loop_roofline"].items()
+                              if k in ("t_roof_ms", "frac", "frac_of_sustained", "frac_of_burst", "frac_of_nominal")},
+            "kv_bytes_peak": line["kv_bytes"]["peak"], "kv_bytes_full_cache": line["kv_bytes"]["full_cache"],
+            "full_cache_run_ms": round(full["ms_per_step"], 4),
+            "speedup_vs_full_cache": round(full["speedup_of_budgeted_run"], 4),
+            "sm_mhz": line["clocks"]["sm_mhz"], "clock_reasons": line["clocks"]["reasons"]}), flush=True)
+
+
+def spawn_ranks(n: int) -> int:
+    """Started plainly with --gpus N > 1: run the same command as N ranks, one per GPU."""
+    have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+    if have < n:
+        print(f"bench.py --gpus {n} needs {n} GPUs on this node; {have} visible", file=sys.stderr)
+        return 2
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -628,6 +708,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3)
+    ap.add_argument("--budget-frac", type=float, default=None, help="point of the budget sweep of configs 2 and 4")
+    ap.add_argument("--alpha", type=float, default=None, help="contextual share of config 4's sweep")
+    ap.add_argument("--sweep", action="store_true",
+                    help="every workload and sweep point, one compact JSON line each, instead of the default loop")
     ap.add_argument("--layers", type=int, default=0, help="restrict the stack (debugging only)")
     ap.add_argument("--oracle-pairs", type=int, default=32)
     ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of graph replays")
@@ -644,8 +728,16 @@ def main():
     ap.add_argument("--head-variance", action="store_true",
                     help="time the attention-variance pass of the offline head classification instead of the loop")
     args = ap.parse_args()
+    args.quiet = False
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.head_variance:
+    world_env = os.environ.get("WORLD_SIZE")
+    if world_env is None and args.gpus > 1 and args.impl == "ours":
+        sys.exit(spawn_ranks(args.gpus))
+    if world_env is not None and int(world_env) != args.gpus and args.impl == "ours":
+        sys.exit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world_env}")
+    if args.sweep:
+        run_sweep(args)
+    elif args.head_variance:
         run_head_variance(args)
     elif args.impl == "reference":
         run_reference(args)

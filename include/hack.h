@@ -253,6 +253,14 @@ HACK_API hack_status_t hack_stage_times(hack_cache_t* cache, double* ms, uint64_
 /* Synchronises `stream`, then reports the device status word: HACK_OK, or HACK_ERR_TIMEOUT if a
  * bounded device-side wait gave up (the word is cleared by the call). */
 HACK_API hack_status_t hack_poll_status(hack_cache_t* cache, void* stream);
+/* Limit, in SM clock cycles, of every bounded device-side wait (mbarrier waits of the tensor-core
+ * kernels) in launches made through this cache from now on; 0 restores the default of about one
+ * second.  A wait that outlasts the limit raises the status word (hack_poll_status then returns
+ * HACK_ERR_TIMEOUT), the CTA drains what it has in flight, frees its tensor memory and returns; the
+ * results of that launch are undefined and the cache should be reset.  Meant for tests of that path
+ * (a limit of a few cycles makes the first wait that is not already satisfied give up) and for
+ * callers that want a tighter bound than a second.  INVALID_ARG for a negative limit. */
+HACK_API hack_status_t hack_set_wait_limit(hack_cache_t* cache, int64_t cycles);
 /* Text of the calling thread's last error; never NULL. */
 HACK_API const char* hack_last_error(void);
 

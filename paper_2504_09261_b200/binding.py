@@ -24,7 +24,8 @@ EXPORTS = (
     "hack_step_info", "hack_score", "hack_select", "hack_compact", "hack_attend", "hack_attend_variance",
     "hack_classify_heads", "hack_scale_step",
     "hack_scale_step_host", "hack_score_noalloc", "hack_get_lengths", "hack_read_head", "hack_kv_bytes",
-    "hack_launch_count", "hack_stage_timing", "hack_stage_times", "hack_poll_status", "hack_last_error",
+    "hack_launch_count", "hack_stage_timing", "hack_stage_times", "hack_poll_status", "hack_set_wait_limit",
+    "hack_last_error",
 )
 
 
@@ -86,6 +87,7 @@ def _load() -> C.CDLL:
         "hack_kv_bytes": [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)],
         "hack_launch_count": [vp, C.POINTER(C.c_uint64)],
         "hack_poll_status": [vp, vp],
+        "hack_set_wait_limit": [vp, C.c_int64],
         "hack_stage_timing": [vp, i32],
         "hack_stage_times": [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)],
     }
@@ -244,6 +246,9 @@ class HackCache:
         _check(lib.hack_stage_times(self._h, ms, n))
         names = ("score", "select", "compact", "attend")
         return {k: (ms[i], n[i]) for i, k in enumerate(names)}
+
+    def hack_set_wait_limit(self, cycles: int) -> None:
+        _check(lib.hack_set_wait_limit(self._h, cycles))
 
     def hack_poll_status(self, stream=None) -> None:
         _check(lib.hack_poll_status(self._h, _ptr(stream)))

@@ -25,6 +25,16 @@
 // TMEM.  K tiles are K-major operands, V tiles MN-major operands, both 128-byte swizzled as TMA
 // writes them.  Softmax keeps a running maximum that is only raised (and O rescaled in TMEM) when
 // a row's maximum grows by more than 2^32, so rescaling is rare after the first tile.
+// (Tried and dropped: logits in two buffers of 64 keys per tile, so that the next Q K^T product
+// runs under the softmax.  The 128 x 64 x 16 MMA re-reads the whole Q operand from shared memory
+// for half the keys and takes nearly as long as the 128 x 128 x 16 one: the last-scale launch of the
+// 10 521-token workload went from 0.233 to 0.301 ms.)
+// The keys and values of a head come in two segments: len_a rows of the head's cache, then len_b
+// rows of the new scale taken straight from the caller's K/V tensors (second pair of tensor maps).
+// Heads that keep the whole new scale (steps without eviction; structural heads, whose latest scale
+// is protected, Eq. 11) are served that way before the new rows are in the cache: the append
+// (Eq. 3) is done by warps 2-3 of the same CTAs, global to global, each CTA of a head taking a
+// slice of the rows; nothing in this launch reads the rows they write.
 // Every mbarrier wait is bounded; on expiry the CTA raises the status word, drains what it has in
 // flight, frees its TMEM and returns.
 #include <cuda.h>
@@ -42,17 +52,25 @@ constexpr int kBN = 128;                 // cache rows per K/V tile
 constexpr int kThreadsTc = 384;
 constexpr int kMmaWarp = 0, kProducerWarp = 1;   // the issuer is the oldest warp of its scheduler
 constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // 2*128*224 + 128*56 = 384*168 registers
-constexpr int kPolyOf8 = 0;              // pairs out of 8 whose 2^x runs on the FMA pipe
+constexpr int kPolyOf8 = 2;              // pairs out of 8 whose 2^x runs on the FMA pipe
 constexpr int kKStages = 2;
 constexpr int kVStages = 2;
 constexpr uint32_t kSpinLimit = 1u << 22;          // polls while draining after an abort
-constexpr long long kWaitCycles = 2000000000ll;    // about one second: no wait here is legitimately longer
 constexpr float kRescaleThreshold = 32.0f;   // log2 units: p <= 2^32, far inside the bf16 / fp32 range
 
 struct TcParams {
   int n_heads, n_new, n_pairs;           // n_pairs: CTAs per head
   int tiles_per_cta;                     // 2, or 1 when the grid would not fill the GPU otherwise
-  int kept[2];
+  int len_a[2], len_b[2];                // per head type: rows read from the cache, then from the caller's K/V
+  int append_new;                        // heads with len_b > 0 also store those rows behind their len_a cache rows
+  int pos_base;                          // global position of the new scale's first token
+  int head_dim_pieces;                   // 16-byte pieces per row
+  long long wait_cycles;                 // limit of every mbarrier wait
+  uint4* k_plane;                        // cache planes of this layer (append only)
+  uint4* v_plane;
+  int32_t* pos_plane;
+  const uint4* k_new;                    // the caller's K/V (append only)
+  const uint4* v_new;
   float scale_log2;                      // sm_scale * log2(e)
   const uint8_t* is_ctx;
   const int32_t* row_off;
@@ -72,7 +90,8 @@ struct Bars {
   int abort_flag;
 };
 
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Bars* b, int* status, int code) {
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Bars* b, int* status, int code,
+                                         long long limit) {
   const uint32_t addr = smem_u32(bar);
   if (mbar_try_wait(addr, parity)) return true;
   const long long t0 = clock64();
@@ -80,7 +99,7 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Bars* b
     if (mbar_try_wait(addr, parity)) return true;
     if ((it & 63u) == 63u) {
       if (*reinterpret_cast<volatile int*>(&b->abort_flag)) return false;
-      if (clock64() - t0 > kWaitCycles) break;
+      if (clock64() - t0 > limit) break;
     }
   }
   *reinterpret_cast<volatile int*>(&b->abort_flag) = 1;
@@ -91,7 +110,8 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, Bars* b
 template <int D>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                 const __grid_constant__ CUtensorMap tm_v, const TcParams p) {
+                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kn,
+                 const __grid_constant__ CUtensorMap tm_vn, const TcParams p) {
   constexpr int SUB = D / 64;                       // 64-column (128-byte) sub-tiles per row
   constexpr uint32_t SUB_BYTES = kBN * 128;         // one sub-tile: 128 rows x 128 bytes
   constexpr uint32_t TILE_BYTES = SUB * SUB_BYTES;
@@ -109,13 +129,21 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bh = p.head_order[blockIdx.x / p.n_pairs];
   const int pair = blockIdx.x % p.n_pairs;
-  const int len = p.kept[p.is_ctx[bh % p.n_heads]];
-  const int nblk = (len + kBN - 1) / kBN;
+  const int type = p.is_ctx[bh % p.n_heads];
+  const int len_a = p.len_a[type], len_b = p.len_b[type];
+  const int nblk_a = (len_a + kBN - 1) / kBN;
+  const int nblk = nblk_a + (len_b + kBN - 1) / kBN;      // >= 1: a head never attends over nothing
   const int q0 = pair * p.tiles_per_cta * kBM;
   const int ntile = (p.tiles_per_cta == 2 && q0 + kBM < p.n_new) ? 2 : 1;
 
   const int qrow = bh * p.n_new + q0;
   const int krow = p.row_off[bh];
+  const int nrow = bh * p.n_new;
+  const long long wlim = p.wait_cycles;
+  // K / V tile j of this head: which tensor it comes from and its first row there
+  auto k_src = [&](int j) { return j < nblk_a ? &tm_k : &tm_kn; };
+  auto v_src = [&](int j) { return j < nblk_a ? &tm_v : &tm_vn; };
+  auto tile_row = [&](int j) { return j < nblk_a ? krow + j * kBN : nrow + (j - nblk_a) * kBN; };
   if (warp == kProducerWarp && lane == 0) {
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(&bars->q_full[t]), 1);
@@ -135,6 +163,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     prefetch_tensormap(&tm_q);
     prefetch_tensormap(&tm_k);
     prefetch_tensormap(&tm_v);
+    if (len_b > 0) {
+      prefetch_tensormap(&tm_kn);
+      prefetch_tensormap(&tm_vn);
+    }
     pdl_wait();
     for (int t = 0; t < ntile; ++t) {
       const uint32_t bar = smem_u32(&bars->q_full[t]);
@@ -143,9 +175,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         tma_load_2d(q_sm + t * TILE_BYTES + c * SUB_BYTES, &tm_q, c * 64, qrow + t * kBM, bar);
     }
     mbar_expect_tx(smem_u32(&bars->k_full[0]), TILE_BYTES);
-    for (int c = 0; c < SUB; ++c) tma_load_2d(k_sm + c * SUB_BYTES, &tm_k, c * 64, krow, smem_u32(&bars->k_full[0]));
+    for (int c = 0; c < SUB; ++c) tma_load_2d(k_sm + c * SUB_BYTES, k_src(0), c * 64, tile_row(0), smem_u32(&bars->k_full[0]));
     mbar_expect_tx(smem_u32(&bars->v_full[0]), TILE_BYTES);
-    for (int c = 0; c < SUB; ++c) tma_load_2d(v_sm + c * SUB_BYTES, &tm_v, c * 64, krow, smem_u32(&bars->v_full[0]));
+    for (int c = 0; c < SUB; ++c) tma_load_2d(v_sm + c * SUB_BYTES, v_src(0), c * 64, tile_row(0), smem_u32(&bars->v_full[0]));
   }
   if (warp == kMmaWarp) {
     tmem_alloc(smem_u32(&bars->tmem_base), 512);
@@ -159,6 +191,31 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   if (warp == 2 || warp == 3) {
     reg_dec<kOtherRegs>();
+    if (p.append_new && len_b > 0) {
+      // Eq. 3 for this head: the new scale's rows go behind the len_a cache rows.  The CTAs of the
+      // head share the rows; whole rows of K and V, 16 bytes per thread, four loads in flight.
+      const int per_cta = (len_b + p.n_pairs - 1) / p.n_pairs;
+      const int r0 = pair * per_cta, r1 = min(len_b, r0 + per_cta);
+      const int pieces = p.head_dim_pieces;
+      const int t = tid - 64;                                   // 0..63
+      const size_t src0 = (size_t)nrow * pieces, dst0 = (size_t)(krow + len_a) * pieces;
+      const int n = max(r1 - r0, 0) * pieces;
+      const int first = r0 * pieces;
+      for (int i0 = 0; i0 < n; i0 += 64 * 4) {
+        uint4 kv[4], vv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * 64 + t;
+          if (i < n) { kv[u] = p.k_new[src0 + first + i]; vv[u] = p.v_new[src0 + first + i]; }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u * 64 + t;
+          if (i < n) { p.k_plane[dst0 + first + i] = kv[u]; p.v_plane[dst0 + first + i] = vv[u]; }
+        }
+      }
+      for (int r = r0 + t; r < r1; r += 64) p.pos_plane[krow + len_a + r] = p.pos_base + r;
+    }
   } else if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ TMA producer
     reg_dec<kOtherRegs>();
@@ -168,22 +225,22 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       for (int j = 1; j < nblk && ok; ++j) {
         {
           const int s = j % kKStages;
-          ok = wait_bar(&bars->k_empty[s], ((j / kKStages) & 1) ^ 1, bars, p.status, 1);
+          ok = wait_bar(&bars->k_empty[s], ((j / kKStages) & 1) ^ 1, bars, p.status, 1, wlim);
           if (!ok) break;
           const uint32_t bar = smem_u32(&bars->k_full[s]);
           mbar_expect_tx(bar, TILE_BYTES);
           for (int c = 0; c < SUB; ++c)
-            tma_load_2d(k_sm + s * TILE_BYTES + c * SUB_BYTES, &tm_k, c * 64, krow + j * kBN, bar);
+            tma_load_2d(k_sm + s * TILE_BYTES + c * SUB_BYTES, k_src(j), c * 64, tile_row(j), bar);
           ++k_issued;
         }
         {
           const int s = j % kVStages;
-          ok = wait_bar(&bars->v_empty[s], ((j / kVStages) & 1) ^ 1, bars, p.status, 2);
+          ok = wait_bar(&bars->v_empty[s], ((j / kVStages) & 1) ^ 1, bars, p.status, 2, wlim);
           if (!ok) break;
           const uint32_t bar = smem_u32(&bars->v_full[s]);
           mbar_expect_tx(bar, TILE_BYTES);
           for (int c = 0; c < SUB; ++c)
-            tma_load_2d(v_sm + s * TILE_BYTES + c * SUB_BYTES, &tm_v, c * 64, krow + j * kBN, bar);
+            tma_load_2d(v_sm + s * TILE_BYTES + c * SUB_BYTES, v_src(j), c * 64, tile_row(j), bar);
           ++v_issued;
         }
       }
@@ -220,8 +277,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         else mma_ss_chain4(tmem + S_COL + t * kBN, q_desc[t], kd, IDESC_S, 0);
         mma_commit(smem_u32(&bars->s_full[t]));
       };
-      for (int t = 0; t < ntile && ok; ++t) ok = wait_bar(&bars->q_full[t], 0, bars, p.status, 3);
-      if (ok) ok = wait_bar(&bars->k_full[0], 0, bars, p.status, 4);
+      for (int t = 0; t < ntile && ok; ++t) ok = wait_bar(&bars->q_full[t], 0, bars, p.status, 3, wlim);
+      if (ok) ok = wait_bar(&bars->k_full[0], 0, bars, p.status, 4, wlim);
       if (ok) {
         tc_fence_after();
         for (int t = 0; t < ntile; ++t) issue_s(t, 0);
@@ -233,19 +290,19 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         for (int t = 0; t < ntile && ok; ++t) {
           // the probabilities arrive in two halves of 64 keys, so that the second MMA starts while
           // the softmax is still working on the second half
-          ok = wait_bar(&bars->p_full[t][0], j & 1, bars, p.status, 5);
-          if (ok && t == 0) ok = wait_bar(&bars->v_full[vs], (j / kVStages) & 1, bars, p.status, 6);
+          ok = wait_bar(&bars->p_full[t][0], j & 1, bars, p.status, 5, wlim);
+          if (ok && t == 0) ok = wait_bar(&bars->v_full[vs], (j / kVStages) & 1, bars, p.status, 6, wlim);
           if (!ok) break;
           tc_fence_after();
           mma_ts_chain4(tmem + O_COL + t * D, tmem + S_COL + t * kBN, vd, IDESC_PV, j > 0);
-          ok = wait_bar(&bars->p_full[t][1], j & 1, bars, p.status, 5);
+          ok = wait_bar(&bars->p_full[t][1], j & 1, bars, p.status, 5, wlim);
           if (!ok) break;
           tc_fence_after();
           mma_ts_chain4(tmem + O_COL + t * D, tmem + S_COL + t * kBN + 32, vd + 4 * 128, IDESC_PV, 1);
           if (t == ntile - 1) mma_commit(smem_u32(&bars->v_empty[vs]));
           if (j + 1 < nblk) {
             if (t == 0) {
-              ok = wait_bar(&bars->k_full[(j + 1) % kKStages], ((j + 1) / kKStages) & 1, bars, p.status, 7);
+              ok = wait_bar(&bars->k_full[(j + 1) % kKStages], ((j + 1) / kKStages) & 1, bars, p.status, 7, wlim);
               if (!ok) break;
               tc_fence_after();
             }
@@ -275,14 +332,15 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       float m_used = -INFINITY, l = 0.f;
       bool ok = true;
       for (int j = 0; j < nblk; ++j) {
-        ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[t], j & 1, bars, p.status, 8));
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->s_full[t], j & 1, bars, p.status, 8, wlim));
         if (!ok) break;
         tc_fence_after();
         uint32_t sr[kBN];
 #pragma unroll
         for (int ch = 0; ch < kBN / 32; ++ch) tmem_ld32(s_addr + ch * 32, sr + ch * 32);
         tmem_wait_ld();
-        const int valid = len - j * kBN;           // >= 1; < 128 only in the last tile
+        // live keys of this tile: fewer than 128 only in the last tile of either segment
+        const int valid = j < nblk_a ? len_a - j * kBN : len_b - (j - nblk_a) * kBN;
         if (valid < kBN) {
 #pragma unroll
           for (int i = 0; i < kBN; ++i)
@@ -344,13 +402,23 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         const float2 sum2 = add2(add2(sum4[0], sum4[1]), add2(sum4[2], sum4[3]));
         l += sum2.x + sum2.y;
+        {
+          // The second MMA sees the probabilities rounded to bf16, the row sum does not.  With the
+          // lazily raised reference maximum even a dominant key's probability is no power of two,
+          // and its rounding error (up to 2^-9 of an output that can reach 4) would pass straight
+          // into O.  The tile's largest probability is therefore entered into the sum as rounded,
+          // which makes the weight of a dominant key exact; what is left is bounded by the weight
+          // of the other keys.  Same instructions as in the loop above, hence the same bits.
+          const float p_top = ex2(fmaf(mx, c, nmc2.x));
+          l += __bfloat162float(__float2bfloat16_rn(p_top)) - p_top;
+        }
         tmem_st32(s_addr + 32, pk + 32);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t][1]));
       }
-      if (ok) ok = __all_sync(0xffffffffu, wait_bar(&bars->o_final[t], 0, bars, p.status, 9));
+      if (ok) ok = __all_sync(0xffffffffu, wait_bar(&bars->o_final[t], 0, bars, p.status, 9, wlim));
       if (ok) {
         tc_fence_after();
         const int row = q0 + t * kBM + r;
@@ -425,18 +493,45 @@ bool make_rows_map(void* out_map, const void* base, uint64_t rows, int head_dim)
 }
 
 int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
-                     const void* q, void* out, float* row_stats, cudaStream_t st) {
+                     const void* q, void* out, float* row_stats, const void* k_new, const void* v_new,
+                     cudaStream_t st) {
   CUtensorMap tm_q;
-  if (!make_rows_map(&tm_q, q, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) return -1;
+  if (!make_rows_map(&tm_q, q, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) {
+    set_error("attention: cuTensorMapEncodeTiled failed for the queries");
+    return -1;
+  }
   TcParams p;
   p.n_heads = a.n_heads;
   p.n_new = a.n_new;
   // one query tile per CTA while that still fits one wave: twice the CTAs, no idle SMs
   const int n_tiles = (a.n_new + kBM - 1) / kBM;
-  p.tiles_per_cta = n_tiles * a.batch * a.n_heads <= 148 ? 1 : 2;
+  p.tiles_per_cta = n_tiles * a.batch * a.n_heads <= sm_count() ? 1 : 2;
   p.n_pairs = (n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
-  p.kept[0] = a.kept[0];
-  p.kept[1] = a.kept[1];
+  const CUtensorMap& tk = *static_cast<const CUtensorMap*>(k_map);
+  const CUtensorMap& tv = *static_cast<const CUtensorMap*>(v_map);
+  CUtensorMap tm_kn = tk, tm_vn = tv;       // placeholders unless a head type reads the caller's rows
+  p.append_new = 0;
+  for (int t = 0; t < 2; ++t) {
+    const bool from_caller = k_new && v_new && a.seg_new[t];
+    p.len_b[t] = from_caller ? a.n_new : 0;
+    p.len_a[t] = a.kept[t] - p.len_b[t];
+    if (from_caller) p.append_new = 1;
+  }
+  if (p.append_new) {
+    const uint64_t rows = (uint64_t)a.batch * a.n_heads * a.n_new;
+    if (!make_rows_map(&tm_kn, k_new, rows, a.head_dim) || !make_rows_map(&tm_vn, v_new, rows, a.head_dim)) {
+      set_error("attention: cuTensorMapEncodeTiled failed for the new scale's keys or values");
+      return -1;
+    }
+  }
+  p.pos_base = a.pos_base;
+  p.head_dim_pieces = a.head_dim * 2 / 16;
+  p.wait_cycles = a.wait_cycles;
+  p.k_plane = static_cast<uint4*>(a.k_plane);
+  p.v_plane = static_cast<uint4*>(a.v_plane);
+  p.pos_plane = a.pos_plane;
+  p.k_new = static_cast<const uint4*>(k_new);
+  p.v_new = static_cast<const uint4*>(v_new);
   p.scale_log2 = a.sm_scale * 1.4426950408889634f;
   p.is_ctx = a.is_ctx;
   p.row_off = a.row_off;
@@ -445,15 +540,13 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
   p.row_stats = row_stats;
   p.status = a.status;
   const int grid = p.n_pairs * a.batch * a.n_heads;
-  const CUtensorMap& tk = *static_cast<const CUtensorMap*>(k_map);
-  const CUtensorMap& tv = *static_cast<const CUtensorMap*>(v_map);
   if (a.head_dim == 128) {
-    allow_dynamic_smem(attend_tc_kernel<128>, tc_smem_bytes<128>());
-    launch_k(attend_tc_kernel<128>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, p);
+    if (!allow_dynamic_smem(attend_tc_kernel<128>, tc_smem_bytes<128>())) return -1;
+    launch_k(attend_tc_kernel<128>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, tm_kn, tm_vn, p);
   } else {
-    allow_dynamic_smem(attend_tc_kernel<64>, tc_smem_bytes<128>());
+    if (!allow_dynamic_smem(attend_tc_kernel<64>, tc_smem_bytes<128>())) return -1;
     // the larger request keeps it at one CTA per SM (the kernel owns all 512 TMEM columns)
-    launch_k(attend_tc_kernel<64>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, p);
+    launch_k(attend_tc_kernel<64>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, tm_kn, tm_vn, p);
   }
   return launched(1);
 }

@@ -27,7 +27,6 @@ using namespace ptx;
 constexpr int kVarThreads = 192;
 constexpr int kVarTile = 128;            // keys per CTA, queries per tile
 constexpr int kQStages = 2;             // 96 KB of tiles at head_dim 128: two CTAs per SM
-constexpr long long kVarWaitCycles = 2000000000ll;   // about one second
 constexpr uint32_t kVarDrainSpins = 1u << 22;
 
 struct VarBars {
@@ -39,14 +38,14 @@ struct VarBars {
   int abort_flag;
 };
 
-__device__ __forceinline__ bool var_wait(uint64_t* bar, uint32_t parity, VarBars* b, int* status, int code) {
+__device__ __forceinline__ bool var_wait(uint64_t* bar, uint32_t parity, VarBars* b, int* status, int code, long long limit) {
   const uint32_t addr = smem_u32(bar);
   const long long t0 = clock64();
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(addr, parity)) return true;
     if ((it & 63u) == 63u) {
       if (*reinterpret_cast<volatile int*>(&b->abort_flag)) return false;
-      if (clock64() - t0 > kVarWaitCycles) break;
+      if (clock64() - t0 > limit) break;
     }
   }
   *reinterpret_cast<volatile int*>(&b->abort_flag) = 1;
@@ -115,7 +114,7 @@ attn_colstats_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       bool ok = true;
       for (int t = 0; t < n_qt; ++t) {
         const int s = t % kQStages;
-        ok = var_wait(&bars->q_empty[s], ((t / kQStages) & 1) ^ 1, bars, a.status, 31);
+        ok = var_wait(&bars->q_empty[s], ((t / kQStages) & 1) ^ 1, bars, a.status, 31, a.wait_cycles);
         if (!ok) break;
         const uint32_t bar = smem_u32(&bars->q_full[s]);
         mbar_expect_tx(bar, TILE_BYTES);
@@ -137,11 +136,11 @@ attn_colstats_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     if (lane == 0) {
       constexpr uint32_t IDESC = idesc_bf16_f32(kVarTile, kVarTile, 0);      // A = keys, B = queries, both K-major
       const uint64_t k_desc = smem_desc_sw128(k_sm, 16, 1024);
-      bool ok = var_wait(&bars->k_full, 0, bars, a.status, 32);
+      bool ok = var_wait(&bars->k_full, 0, bars, a.status, 32, a.wait_cycles);
       for (int t = 0; t < n_qt && ok; ++t) {
         const int s = t % kQStages, b = t & 1;
-        ok = var_wait(&bars->q_full[s], (t / kQStages) & 1, bars, a.status, 33);
-        if (ok) ok = var_wait(&bars->acc_free[b], ((t >> 1) & 1) ^ 1, bars, a.status, 34);
+        ok = var_wait(&bars->q_full[s], (t / kQStages) & 1, bars, a.status, 33, a.wait_cycles);
+        if (ok) ok = var_wait(&bars->acc_free[b], ((t >> 1) & 1) ^ 1, bars, a.status, 34, a.wait_cycles);
         if (!ok) break;
         tc_fence_after();
         const uint64_t q_desc = smem_desc_sw128(q_sm + s * TILE_BYTES, 16, 1024);
@@ -176,8 +175,10 @@ attn_colstats_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         stat[b][ct] = st;
       }
       var_consumer_sync();
-      ok = __all_sync(0xffffffffu, var_wait(&bars->acc_full[b], (t >> 1) & 1, bars, a.status, 35));
-      if (!ok) break;
+      // a warp whose wait gave up keeps walking the loop, so that it still meets the other consumers
+      // on the named barrier above and after the loop; it only stops touching the accumulators
+      if (ok) ok = __all_sync(0xffffffffu, var_wait(&bars->acc_full[b], (t >> 1) & 1, bars, a.status, 35, a.wait_cycles));
+      if (!ok) continue;
       tc_fence_after();
 #pragma unroll
       for (int ch = 0; ch < kVarTile / 32; ++ch) {
@@ -210,7 +211,7 @@ attn_colstats_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) var += __shfl_xor_sync(0xffffffffu, var, o);
-    if (lane == 0) red[warp - 2] = var;
+    if (lane == 0) red[warp - 2] = ok ? var : NAN;           // a warp that gave up poisons the block's sum
     var_consumer_sync();
     if (ct == 0 && ok) block_var[(size_t)bh * max_blocks + kb] = (red[0] + red[1]) + (red[2] + red[3]);
   }
@@ -247,7 +248,10 @@ size_t var_smem_bytes() {
 int launch_attention_variance(const StepArgs& a, const void* q, const float* row_stats, float* block_var,
                               int max_blocks, float* sigma, cudaStream_t st) {
   CUtensorMap tm_q;
-  if (!make_rows_map(&tm_q, q, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) return -1;
+  if (!make_rows_map(&tm_q, q, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) {
+    set_error("attention variance: cuTensorMapEncodeTiled failed for the queries");
+    return -1;
+  }
   const CUtensorMap& tk = *static_cast<const CUtensorMap*>(a.k_map);
   const int bh = a.batch * a.n_heads;
   const int longest = a.kept[0] > a.kept[1] ? a.kept[0] : a.kept[1];
@@ -258,10 +262,10 @@ int launch_attention_variance(const StepArgs& a, const void* q, const float* row
   }
   const dim3 grid(n_blocks, bh);
   if (a.head_dim == 128) {
-    allow_dynamic_smem(attn_colstats_kernel<128>, var_smem_bytes<128>());
+    if (!allow_dynamic_smem(attn_colstats_kernel<128>, var_smem_bytes<128>())) return -1;
     launch_k(attn_colstats_kernel<128>, grid, kVarThreads, var_smem_bytes<128>(), st, tm_q, tk, a, row_stats, block_var, max_blocks);
   } else {
-    allow_dynamic_smem(attn_colstats_kernel<64>, var_smem_bytes<64>());
+    if (!allow_dynamic_smem(attn_colstats_kernel<64>, var_smem_bytes<64>())) return -1;
     launch_k(attn_colstats_kernel<64>, grid, kVarThreads, var_smem_bytes<64>(), st, tm_q, tk, a, row_stats, block_var, max_blocks);
   }
   launch_k(attn_variance_finish_kernel, bh, 32, 0, st, a, block_var, max_blocks, sigma);

@@ -24,8 +24,9 @@ constexpr int kThreads = 256;
 constexpr int kMoveUnroll = 16;       // rows in flight per thread while moving stored rows
 constexpr int kCopyUnroll = 8;        // rows in flight per thread while copying new rows
 
-// Number of list entries below `stored` (the list is ascending), found by the whole CTA with two
-// rounds of probes.
+// Number of list entries below `stored` (the list is ascending), found by the whole CTA: a round
+// of probes finds the block of `step` entries that holds the boundary, then that block is counted
+// (in slices of kThreads entries, so that any list length is served).
 __device__ __forceinline__ int count_old(const int32_t* list, int n_keep, int stored) {
   const int tid = threadIdx.x;
   const int step = (n_keep + kThreads - 1) / kThreads;
@@ -34,8 +35,13 @@ __device__ __forceinline__ int count_old(const int32_t* list, int n_keep, int st
   const bool below = tid * step < n_keep && list[p] < stored;
   const int full_blocks = __syncthreads_count(below);      // blocks that lie entirely below
   const int lo = full_blocks * step;
-  const bool below2 = tid < step && lo + tid < n_keep && list[lo + tid] < stored;
-  return lo + __syncthreads_count(below2);
+  int n = lo;
+  for (int i0 = 0; i0 < step; i0 += kThreads) {
+    const int i = i0 + tid;
+    const bool below2 = i < step && lo + i < n_keep && list[lo + i] < stored;
+    n += __syncthreads_count(below2);
+  }
+  return n;
 }
 
 // PIECES: 16-byte pieces per row handled by one CTA (64-byte slices measured best: narrower ones
@@ -104,6 +110,7 @@ compact_copy_kernel(const StepArgs a, const int32_t* __restrict__ idx, const uin
   pdl_wait();
   const int bh = blockIdx.z;
   const int ctx = a.is_ctx[bh % a.n_heads];
+  if (a.seg_new[ctx]) return;                      // the attention launch appends this type's new rows
   const int stored = a.stored[ctx], n_keep = a.kept[ctx];
   const int32_t* list = idx ? idx + (size_t)bh * a.kept_stride : nullptr;
   const int n_old = list ? a.n_old[bh] : stored;
@@ -151,9 +158,15 @@ int launch_compact(const StepArgs& a, int dtype, const int32_t* idx, int idx_all
   }
   // enough CTAs for the longest list in one pass (n_old is not known here), within a few waves
   const int rows_per_cta = (kThreads / row_pieces) * kCopyUnroll;
-  const int most = idx ? (a.kept[0] > a.kept[1] ? a.kept[0] : a.kept[1]) : a.n_new;
+  if (a.seg_new[0] && a.seg_new[1]) return launched(n);       // no head has rows to copy here
+  int most = a.n_new;
+  if (idx) {
+    most = 0;
+    for (int t = 0; t < 2; ++t)
+      if (!a.seg_new[t] && a.kept[t] > most) most = a.kept[t];
+  }
   int n_copy = (most + rows_per_cta - 1) / rows_per_cta;
-  const int cap = (16 * 148 + 2 * heads - 1) / (2 * heads);
+  const int cap = (16 * sm_count() + 2 * heads - 1) / (2 * heads);
   n_copy = n_copy < 1 ? 1 : (n_copy > cap ? cap : n_copy);
   launch_k(compact_copy_kernel, dim3(n_copy, 2, heads), dim3(kThreads), 0, st, a, idx,
            static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), row_pieces);

@@ -15,16 +15,36 @@ namespace hack {
 static thread_local std::string g_last_error;
 void set_error(const std::string& msg) { g_last_error = msg; }
 
-void allow_dynamic_smem_impl(const void* kern, size_t bytes) {
+bool allow_dynamic_smem_impl(const void* kern, size_t bytes) {
   static std::mutex mu;
   static std::vector<std::pair<const void*, int>> done;        // (kernel, device) pairs already served
   int dev = 0;
   cudaGetDevice(&dev);
   std::lock_guard<std::mutex> lock(mu);
   for (const auto& kd : done)
-    if (kd.first == kern && kd.second == dev) return;
-  cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (kd.first == kern && kd.second == dev) return true;
+  const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e != cudaSuccess) {
+    set_error(std::string("cudaFuncSetAttribute(MaxDynamicSharedMemorySize): ") + cudaGetErrorString(e));
+    return false;
+  }
   done.emplace_back(kern, dev);
+  return true;
+}
+
+int sm_count() {
+  static std::mutex mu;
+  static int count[64] = {0};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64) return 148;
+  std::lock_guard<std::mutex> lock(mu);
+  if (count[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    count[dev] = n;
+  }
+  return count[dev];
 }
 
 bool attend_tc_serves(const StepArgs& a, int dtype) {
@@ -33,7 +53,8 @@ bool attend_tc_serves(const StepArgs& a, int dtype) {
 }
 
 int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st) {
-  if (attend_tc_serves(a, dtype)) return launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, st);
+  if (attend_tc_serves(a, dtype))
+    return launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, nullptr, nullptr, st);
   return launch_attend_simt(a, dtype, q, out, st);
 }
 
@@ -93,6 +114,8 @@ struct hack_cache {
   uint64_t host_calls = 0;
   size_t reserved_bytes = 0, peak_bytes = 0;
   uint64_t launches = 0;
+  long long wait_cycles = hack::kDefaultWaitCycles;   // limit of the kernels' bounded waits
+  bool poisoned = false;                        // a launch failed after part of a step had been enqueued
   // optional per-stage device timing (score, select, compact, attend)
   bool timing = false;
   std::vector<cudaEvent_t> ev_pool;
@@ -166,6 +189,7 @@ hack::StepArgs make_args(const hack_cache* c, int layer, int scale, const hack_s
   a.obs_rows = c->cfg.obs_sampler == HACK_OBS_CALLER ? c->obs_rows + (size_t)scale * hack::kMaxObs : nullptr;
   a.obs_full = c->cfg.obs_sampler == HACK_OBS_FULL;
   a.sm_scale = c->sm_scale;
+  a.wait_cycles = c->wait_cycles;
   a.t_init = c->t_init;
   a.protect_new = (c->cfg.overflow_policy == HACK_OVERFLOW_KEEP_PROTECTED) || scale < c->cfg.n_init_scales;
   a.pos_base = scale == 0 ? 0 : c->t_cum[scale - 1];
@@ -198,8 +222,38 @@ size_t live_bytes(const hack_cache* c) {
   return rows * c->cfg.head_dim * c->elt * 2;
 }
 
+// Makes the cache's device current for the duration of an entry point and puts the caller's back.
+struct DeviceScope {
+  int prev = -1;
+  bool switched = false;
+  cudaError_t err = cudaSuccess;
+  explicit DeviceScope(int want) {
+    err = cudaGetDevice(&prev);
+    if (err == cudaSuccess && prev != want) {
+      err = cudaSetDevice(want);
+      switched = err == cudaSuccess;
+    }
+  }
+  ~DeviceScope() { if (switched) cudaSetDevice(prev); }
+};
+#define HACK_ON_DEVICE(c)                                                                        \
+  DeviceScope dev_scope_((c)->cfg.device);                                                       \
+  if (dev_scope_.err != cudaSuccess) {                                                           \
+    set_error(std::string("selecting the cache's device: ") + cudaGetErrorString(dev_scope_.err)); \
+    return HACK_ERR_CUDA;                                                                        \
+  }
+
+// A launcher failed after earlier launches of the same step were enqueued: the device-side state
+// of the layer no longer matches the host's plan, so the cache refuses further steps until reset.
+hack_status_t poison(hack_cache* c) {
+  c->poisoned = true;
+  return HACK_ERR_CUDA;   // text recorded by the launcher
+}
+
 hack_status_t check_step(const hack_cache* c, int layer, int scale, int want_phase) {
   if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
+  if (c->poisoned)
+    return fail(HACK_ERR_STATE, "an earlier step failed half way (a kernel launch was refused); call hack_reset before the next image");
   if (layer < 0 || layer >= c->cfg.n_layers) return fail(HACK_ERR_INVALID_ARG, "layer out of range");
   if (scale < 0 || scale >= c->cfg.n_scales) return fail(HACK_ERR_INVALID_ARG, "scale out of range");
   const LayerState& ls = c->layers[layer];
@@ -506,6 +560,7 @@ hack_status_t hack_reset(hack_cache_t* c) {
   if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
   for (auto& ls : c->layers) ls = LayerState();
   c->peak_bytes = 0;
+  c->poisoned = false;
   return HACK_OK;
 }
 
@@ -530,6 +585,7 @@ hack_status_t hack_score(hack_cache_t* c, int32_t layer, int32_t scale, const vo
                          const void* k_new, float* scores, void* stream) {
   hack_status_t s = check_step(c, layer, scale, 0);
   if (s != HACK_OK) return s;
+  HACK_ON_DEVICE(c);
   if (!q || !k_new || !scores) return fail(HACK_ERR_INVALID_ARG, "q, k_new or scores is NULL");
   if (misaligned(q) || misaligned(k_new) || misaligned(scores)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
   hack_step_info_t p;
@@ -538,7 +594,9 @@ hack_status_t hack_score(hack_cache_t* c, int32_t layer, int32_t scale, const vo
     return fail(HACK_ERR_STATE, "HACK_OBS_CALLER: no observation rows were set for this scale (hack_set_obs_rows)");
   const hack::StepArgs a = make_args(c, layer, scale, p);
   StageScope ts(c, (cudaStream_t)stream, 0);
-  const int n = hack::launch_score(a, c->cfg.dtype, q, k_new, scores, c->scratch, (cudaStream_t)stream);
+  int n = c->cfg.dtype == HACK_BF16
+              ? hack::launch_compress_cluster(a, q, k_new, nullptr, scores, nullptr, (cudaStream_t)stream) : 0;
+  if (n == 0) n = hack::launch_score(a, c->cfg.dtype, q, k_new, scores, c->scratch, (cudaStream_t)stream);
   if (n < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
   ts.done(n);
   c->launches += n;
@@ -549,6 +607,7 @@ hack_status_t hack_select(hack_cache_t* c, int32_t layer, int32_t scale, const f
                           int32_t* idx, int32_t* kept_out, void* stream) {
   hack_status_t s = check_step(c, layer, scale, 0);
   if (s != HACK_OK) return s;
+  HACK_ON_DEVICE(c);
   if (!scores || !idx) return fail(HACK_ERR_INVALID_ARG, "scores or idx is NULL");
   hack_step_info_t p;
   plan_step(c, c->layers[layer], scale, &p);
@@ -584,6 +643,7 @@ hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const 
                            const void* k_new, const void* v_new, void* stream) {
   hack_status_t s = check_step(c, layer, scale, 0);
   if (s != HACK_OK) return s;
+  HACK_ON_DEVICE(c);
   if (!idx || !k_new || !v_new) return fail(HACK_ERR_INVALID_ARG, "idx, k_new or v_new is NULL");
   if (misaligned(k_new) || misaligned(v_new)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
   hack_step_info_t p;
@@ -598,8 +658,11 @@ hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const 
   return HACK_OK;
 }
 
+// k_new / v_new / seg_new: fused step only; head types flagged in seg_new have their new rows read
+// from the caller's tensors and appended by the attention kernel itself.
 static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void* q, void* out, float* sigma,
-                                 cudaStream_t st) {
+                                 cudaStream_t st, const void* k_new = nullptr, const void* v_new = nullptr,
+                                 const int* seg_new = nullptr) {
   // lengths are already those after compaction
   LayerState& ls = c->layers[layer];
   hack_step_info_t p{};
@@ -607,18 +670,21 @@ static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void
   p.kept_s = ls.len[0];
   p.kept_c = ls.len[1];
   p.n_obs_rows = std::min(c->cfg.n_obs, p.n_new);
-  const hack::StepArgs a = make_args(c, layer, scale, p);
+  hack::StepArgs a = make_args(c, layer, scale, p);
+  if (seg_new) { a.seg_new[0] = seg_new[0]; a.seg_new[1] = seg_new[1]; }
   StageScope ts(c, st, 3);
   int n;
   if (sigma) {
     // Eq. 6 needs the statistics of every softmax row; the tensor-core attention kernel leaves them
     if (!hack::attend_tc_serves(a, c->cfg.dtype))
       return fail(HACK_ERR_UNSUPPORTED, "hack_attend_variance needs a bf16 cache and a scale of at least 32 tokens (128 query rows over all heads)");
-    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, c->attn_row_stats, st);
+    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, c->attn_row_stats, nullptr, nullptr, st);
     if (n >= 0) {
       const int m = hack::launch_attention_variance(a, q, c->attn_row_stats, c->attn_block_var, c->var_blocks, sigma, st);
       n = m < 0 ? m : n + m;
     }
+  } else if (seg_new) {
+    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, k_new, v_new, st);
   } else {
     n = hack::launch_attend(a, c->cfg.dtype, q, out, st);
   }
@@ -633,6 +699,7 @@ static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void
 hack_status_t hack_attend(hack_cache_t* c, int32_t layer, int32_t scale, const void* q, void* out, void* stream) {
   hack_status_t s = check_step(c, layer, scale, 1);
   if (s != HACK_OK) return s;
+  HACK_ON_DEVICE(c);
   if (!q || !out) return fail(HACK_ERR_INVALID_ARG, "q or out is NULL");
   if (misaligned(q) || misaligned(out)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
   return attend_impl(c, layer, scale, q, out, nullptr, (cudaStream_t)stream);
@@ -642,6 +709,7 @@ hack_status_t hack_attend_variance(hack_cache_t* c, int32_t layer, int32_t scale
                                    float* sigma, void* stream) {
   hack_status_t s = check_step(c, layer, scale, 1);
   if (s != HACK_OK) return s;
+  HACK_ON_DEVICE(c);
   if (!q || !out || !sigma) return fail(HACK_ERR_INVALID_ARG, "q, out or sigma is NULL");
   if (misaligned(q) || misaligned(out)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
   return attend_impl(c, layer, scale, q, out, sigma, (cudaStream_t)stream);
@@ -668,6 +736,7 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
                               const void* k, const void* v, void* out, void* stream) {
   hack_status_t s = check_step(c, layer, scale, 0);
   if (s != HACK_OK) return s;
+  HACK_ON_DEVICE(c);
   if (!q || !k || !v || !out) return fail(HACK_ERR_INVALID_ARG, "q, k, v or out is NULL");
   if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(out)) return fail(HACK_ERR_INVALID_ARG, "buffers must be 16-byte aligned");
   cudaStream_t st = (cudaStream_t)stream;
@@ -675,9 +744,23 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
   plan_step(c, c->layers[layer], scale, &p);
   if (c->cfg.obs_sampler == HACK_OBS_CALLER && (p.triggered_c || p.triggered_s) && !c->obs_rows_set[scale])
     return fail(HACK_ERR_STATE, "HACK_OBS_CALLER: no observation rows were set for this scale (hack_set_obs_rows)");
-  const hack::StepArgs a = make_args(c, layer, scale, p);
+  hack::StepArgs a = make_args(c, layer, scale, p);
   const bool any = p.triggered_c || p.triggered_s;
   int n = 0, r;
+  // Tensor-core attention takes the rows of a head type that keeps the whole new scale straight
+  // from the caller's K/V and appends them itself: types that evict nothing in this step, and
+  // structural heads whose latest scale is protected (Eq. 11).  Contextual heads that evict rank the
+  // new rows as well (Eq. 10) and are compacted first.  The final-scale merge keeps the separate
+  // compaction it is wrapped around.
+  const bool merge_step = c->cfg.merge_last && scale == c->cfg.n_scales - 1 && p.triggered_c;
+  int seg_new[2] = {0, 0};
+  const bool fused_append = hack::attend_tc_serves(a, c->cfg.dtype) && !merge_step;
+  if (fused_append) {
+    seg_new[0] = !p.triggered_s || a.protect_new;
+    seg_new[1] = !p.triggered_c;
+    a.seg_new[0] = seg_new[0];
+    a.seg_new[1] = seg_new[1];
+  }
   if (!any && p.n_new <= hack::kSmallQueries) {
     // nothing is evicted and the scale is small: one launch appends and attends
     StageScope ts(c, st, 3);
@@ -690,7 +773,16 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
     ls.next_scale = scale + 1;
     return HACK_OK;
   }
-  if (any) {
+  bool compressed = false;
+  if (any && fused_append) {
+    // score, select and compact in one cluster launch per head (counted with the scoring stage)
+    StageScope ts(c, st, 0);
+    if ((r = hack::launch_compress_cluster(a, q, k, v, nullptr, c->idx, st)) < 0) return HACK_ERR_CUDA;
+    ts.done(r);
+    n += r;
+    compressed = r > 0;
+  }
+  if (any && !compressed) {
     {
       StageScope ts(c, st, 0);
       if ((r = hack::launch_score(a, c->cfg.dtype, q, k, c->scores, c->scratch, st)) < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
@@ -699,46 +791,54 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
     }
     {
       StageScope ts(c, st, 1);
-      if ((r = hack::launch_select(a, c->scores, c->idx, nullptr, st)) < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
+      if ((r = hack::launch_select(a, c->scores, c->idx, nullptr, st)) < 0) return poison(c);
       ts.done(r);
       n += r;
     }
   }
-  {
+  if ((any && !compressed) || !fused_append) {      // a step that only appends needs no launch ahead of the fused attention
     StageScope ts(c, st, 2);
-    if ((r = compact_stage(c, a, p, scale, any ? c->idx : nullptr, any ? 1 : 0, k, v, st)) < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
+    if ((r = compact_stage(c, a, p, scale, any ? c->idx : nullptr, any ? 1 : 0, k, v, st)) < 0) return any ? poison(c) : HACK_ERR_CUDA;
     ts.done(r);
     n += r;
   }
   c->launches += n;
   advance_after_compact(c, layer, p);
-  return attend_impl(c, layer, scale, q, out, nullptr, st);
+  s = attend_impl(c, layer, scale, q, out, nullptr, st, k, v, fused_append ? seg_new : nullptr);
+  if (s == HACK_ERR_CUDA) c->poisoned = true;     // compacted, attention not enqueued
+  return s;
 }
 
 hack_status_t hack_scale_step_host(hack_cache_t* c, int32_t layer, int32_t scale, const void* q_host,
                                    const void* k_host, const void* v_host, void* out_host, void* stream) {
   hack_status_t s = check_step(c, layer, scale, 0);
   if (s != HACK_OK) return s;
+  HACK_ON_DEVICE(c);
   if (!q_host || !k_host || !v_host || !out_host) return fail(HACK_ERR_INVALID_ARG, "a host buffer is NULL");
   cudaStream_t st = (cudaStream_t)stream;
   const size_t full = (size_t)c->cfg.batch * c->cfg.n_heads * c->limits.max_new * c->cfg.head_dim * c->elt;
   if (!c->h2d_stream) {
     // first use: staging sets, the two copy streams and the events that order them
-    bool ok = cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
-    for (int sl = 0; sl < hack_cache::kHostSlots && ok; ++sl) {
-      for (int i = 0; i < 4 && ok; ++i) ok = cudaMalloc(&c->stage[sl][i], full) == cudaSuccess;
-      ok = ok && cudaEventCreateWithFlags(&c->ev_in[sl], cudaEventDisableTiming) == cudaSuccess &&
-           cudaEventCreateWithFlags(&c->ev_step[sl], cudaEventDisableTiming) == cudaSuccess &&
-           cudaEventCreateWithFlags(&c->ev_out[sl], cudaEventDisableTiming) == cudaSuccess;
+    cudaError_t e = cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking);
+    for (int sl = 0; sl < hack_cache::kHostSlots && e == cudaSuccess; ++sl) {
+      for (int i = 0; i < 4 && e == cudaSuccess; ++i) e = cudaMalloc(&c->stage[sl][i], full);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_in[sl], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_step[sl], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_out[sl], cudaEventDisableTiming);
     }
-    if (!ok) {
-      set_error(std::string("staging set-up: ") + cudaGetErrorString(cudaGetLastError()));
-      for (int sl = 0; sl < hack_cache::kHostSlots; ++sl)
+    if (e != cudaSuccess) {
+      set_error(std::string("staging set-up: ") + cudaGetErrorString(e));
+      cudaGetLastError();
+      for (int sl = 0; sl < hack_cache::kHostSlots; ++sl) {
         for (int i = 0; i < 4; ++i) { cudaFree(c->stage[sl][i]); c->stage[sl][i] = nullptr; }
+        if (c->ev_in[sl]) { cudaEventDestroy(c->ev_in[sl]); c->ev_in[sl] = nullptr; }
+        if (c->ev_step[sl]) { cudaEventDestroy(c->ev_step[sl]); c->ev_step[sl] = nullptr; }
+        if (c->ev_out[sl]) { cudaEventDestroy(c->ev_out[sl]); c->ev_out[sl] = nullptr; }
+      }
       if (c->h2d_stream) { cudaStreamDestroy(c->h2d_stream); c->h2d_stream = nullptr; }
       if (c->d2h_stream) { cudaStreamDestroy(c->d2h_stream); c->d2h_stream = nullptr; }
-      return HACK_ERR_OOM;
+      return e == cudaErrorMemoryAllocation ? HACK_ERR_OOM : HACK_ERR_CUDA;
     }
   }
   const int sl = (int)(c->host_calls % hack_cache::kHostSlots);
@@ -789,6 +889,7 @@ hack_status_t hack_read_head(hack_cache_t* c, int32_t layer, int32_t b, int32_t 
   const size_t need = which == 2 ? len * sizeof(int32_t) : len * row_bytes;
   if (bytes < need) return fail(HACK_ERR_INVALID_ARG, "host_out is too small for the stored length");
   const size_t off = c->row_off_host[((size_t)layer * c->cfg.batch + b) * c->cfg.n_heads + h];
+  HACK_ON_DEVICE(c);
   HACK_CUDA(cudaDeviceSynchronize());
   const size_t row = c->layer_row_base[layer] + off;
   if (need == 0) return HACK_OK;
@@ -813,6 +914,7 @@ hack_status_t hack_launch_count(const hack_cache_t* c, uint64_t* launches) {
 
 hack_status_t hack_stage_timing(hack_cache_t* c, int32_t enable) {
   if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
+  HACK_ON_DEVICE(c);
   HACK_CUDA(cudaDeviceSynchronize());
   c->timing = enable != 0;
   c->spans.clear();
@@ -823,6 +925,7 @@ hack_status_t hack_stage_timing(hack_cache_t* c, int32_t enable) {
 
 hack_status_t hack_stage_times(hack_cache_t* c, double* ms, uint64_t* launches) {
   if (!c || !ms || !launches) return fail(HACK_ERR_INVALID_ARG, "cache, ms or launches is NULL");
+  HACK_ON_DEVICE(c);
   HACK_CUDA(cudaDeviceSynchronize());
   for (const auto& sp : c->spans) {
     float t = 0.f;
@@ -836,8 +939,16 @@ hack_status_t hack_stage_times(hack_cache_t* c, double* ms, uint64_t* launches) 
   return HACK_OK;
 }
 
+hack_status_t hack_set_wait_limit(hack_cache_t* c, int64_t cycles) {
+  if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
+  if (cycles < 0) return fail(HACK_ERR_INVALID_ARG, "the wait limit must not be negative");
+  c->wait_cycles = cycles == 0 ? hack::kDefaultWaitCycles : (long long)cycles;
+  return HACK_OK;
+}
+
 hack_status_t hack_poll_status(hack_cache_t* c, void* stream) {
   if (!c) return fail(HACK_ERR_INVALID_ARG, "cache is NULL");
+  HACK_ON_DEVICE(c);
   HACK_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
   int word = 0;
   HACK_CUDA(cudaMemcpy(&word, c->status, sizeof(int), cudaMemcpyDeviceToHost));

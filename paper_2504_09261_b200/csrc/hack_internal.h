@@ -24,6 +24,9 @@ struct StepArgs {
   int cand[2];          // T' = L + N_k
   int kept[2];          // length after the step
   int trig[2];          // compression triggered for this type
+  int seg_new[2];       // tensor-core attention reads this type's new rows from the caller's K/V and
+                        // appends them itself (the type keeps the whole new scale in this step)
+  long long wait_cycles;   // limit of every bounded device-side wait of the step's kernels
   int n_obs_rows;       // min(N_obs, N_k)
   int obs_first, obs_span;      // observation row i = obs_first + floor(i * obs_span / n_obs_rows) ...
   const int32_t* obs_rows;      // ... unless the caller supplied the rows (device, [n_obs_rows])
@@ -79,6 +82,11 @@ int launch_score_tc(const StepArgs& a, const void* q, const void* k_new, float* 
                     cudaStream_t st);
 int launch_select(const StepArgs& a, const float* scores, int32_t* idx, int32_t* kept_out,
                   cudaStream_t st);
+// bf16 caches: scores only (idx == nullptr) or scoring, selection and in-place compaction of the step
+// in one launch of one thread-block cluster per head.  1: launched; 0: the step is outside what the
+// kernel holds, take the separate launches; -1: launch error.
+int launch_compress_cluster(const StepArgs& a, const void* q, const void* k_new, const void* v_new, float* scores,
+                            int32_t* idx, cudaStream_t st);
 // idx == nullptr: every head appends (keeps all candidates).  idx_all != 0: idx rows are valid for
 // heads that are not triggered as well (identity lists written by launch_select).
 int launch_compact(const StepArgs& a, int dtype, const int32_t* idx, int idx_all, const void* k_new,
@@ -88,8 +96,13 @@ int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaSt
 int launch_attend_simt(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st);
 // row_stats (optional, device [b*H, N_k, 2]): per query row the reference maximum m (raw logit
 // units; within the lazy-rescaling margin of the true maximum) and l = sum_j exp2(c (z_j - m)).
+// k_new / v_new (optional): the caller's K/V of this scale; head types with a.seg_new set then attend
+// over [kept - N_k cache rows ; the N_k new rows read from k_new / v_new] and the kernel appends
+// those rows to the cache, so no append or copy launch precedes it for them.
 int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
-                     const void* q, void* out, float* row_stats, cudaStream_t st);
+                     const void* q, void* out, float* row_stats, const void* k_new, const void* v_new,
+                     cudaStream_t st);
+constexpr long long kDefaultWaitCycles = 2000000000ll;   // about one second: no wait is legitimately longer
 // Attention variance per (batch, head) over the compacted cache (Eq. 6) from the row statistics of
 // launch_attend_tc; block_var: device scratch [b*H, max_blocks]; sigma: device [b*H].  bf16 only.
 int launch_attention_variance(const StepArgs& a, const void* q, const float* row_stats, float* block_var,
@@ -106,6 +119,8 @@ constexpr int kSmallQueries = 31;
 constexpr int kTcMinQueries = 32;   // below this the SIMT kernel serves bf16 as well
 
 void set_error(const std::string& msg);
+// Number of SMs of the current device (asked once per device); the grid heuristics size to it.
+int sm_count();
 
 // Every kernel of the step is launched with programmatic stream serialisation: its CTAs may start
 // while the previous kernel of the stream drains, and stop at pdl_wait() until that kernel has
@@ -138,10 +153,11 @@ __device__ __forceinline__ void pdl_wait() {
 
 // Opt-in to more than 48 KB of dynamic shared memory.  The attribute belongs to the (function,
 // device) pair, so it is set once per pair, on the device that is current (thread safe).
-void allow_dynamic_smem_impl(const void* kern, size_t bytes);
+// False (with the error text recorded) if the driver refuses; the pair is then asked again next time.
+bool allow_dynamic_smem_impl(const void* kern, size_t bytes);
 template <typename F>
-inline void allow_dynamic_smem(F* kern, size_t bytes) {
-  allow_dynamic_smem_impl(reinterpret_cast<const void*>(kern), bytes);
+inline bool allow_dynamic_smem(F* kern, size_t bytes) {
+  return allow_dynamic_smem_impl(reinterpret_cast<const void*>(kern), bytes);
 }
 
 // After a kernel launch: n if it was accepted, else -1 with the CUDA error text recorded.

@@ -38,7 +38,6 @@ constexpr int kApplyThreads = 256;
 constexpr int kApplyRowsPerWarp = 8;     // retained rows per warp (64 per CTA)
 constexpr int kApplyChunk = 2048;        // discarded entries staged in shared memory at a time
 constexpr int kApplyHits = 256;          // entries a warp lists before it works them off
-constexpr long long kMergeWaitCycles = 2000000000ll;   // about one second
 constexpr uint32_t kMergeDrainSpins = 1u << 22;
 
 // ---------------------------------------------------------------- complement of the kept list
@@ -141,14 +140,14 @@ struct AssignBars {
   int abort_flag;
 };
 
-__device__ __forceinline__ bool merge_wait(uint64_t* bar, uint32_t parity, AssignBars* b, int* status, int code) {
+__device__ __forceinline__ bool merge_wait(uint64_t* bar, uint32_t parity, AssignBars* b, int* status, int code, long long limit) {
   const uint32_t addr = smem_u32(bar);
   const long long t0 = clock64();
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(addr, parity)) return true;
     if ((it & 63u) == 63u) {
       if (*reinterpret_cast<volatile int*>(&b->abort_flag)) return false;
-      if (clock64() - t0 > kMergeWaitCycles) break;
+      if (clock64() - t0 > limit) break;
     }
   }
   *reinterpret_cast<volatile int*>(&b->abort_flag) = 1;
@@ -215,7 +214,7 @@ merge_assign_kernel(const __grid_constant__ CUtensorMap tm_e, const __grid_const
       bool ok = true;
       for (int t = 0; t < n_kt; ++t) {
         const int s = t % kRing;
-        ok = merge_wait(&bars->k_empty[s], ((t / kRing) & 1) ^ 1, bars, a.status, 41);
+        ok = merge_wait(&bars->k_empty[s], ((t / kRing) & 1) ^ 1, bars, a.status, 41, a.wait_cycles);
         if (!ok) break;
         const uint32_t bar = smem_u32(&bars->k_full[s]);
         mbar_expect_tx(bar, TILE_BYTES);
@@ -236,11 +235,11 @@ merge_assign_kernel(const __grid_constant__ CUtensorMap tm_e, const __grid_const
     if (lane == 0) {
       constexpr uint32_t IDESC = idesc_bf16_f32(kTileM, kTileM, 0);     // A = discarded keys, B = retained keys, K-major
       const uint64_t e_desc = smem_desc_sw128(e_sm, 16, 1024);
-      bool ok = merge_wait(&bars->e_full, 0, bars, a.status, 42);
+      bool ok = merge_wait(&bars->e_full, 0, bars, a.status, 42, a.wait_cycles);
       for (int t = 0; t < n_kt && ok; ++t) {
         const int s = t % kRing, b = t & 1;
-        ok = merge_wait(&bars->k_full[s], (t / kRing) & 1, bars, a.status, 43);
-        if (ok) ok = merge_wait(&bars->acc_free[b], ((t >> 1) & 1) ^ 1, bars, a.status, 44);
+        ok = merge_wait(&bars->k_full[s], (t / kRing) & 1, bars, a.status, 43, a.wait_cycles);
+        if (ok) ok = merge_wait(&bars->acc_free[b], ((t >> 1) & 1) ^ 1, bars, a.status, 44, a.wait_cycles);
         if (!ok) break;
         tc_fence_after();
         const uint64_t k_desc = smem_desc_sw128(k_sm + s * TILE_BYTES, 16, 1024);
@@ -270,8 +269,10 @@ merge_assign_kernel(const __grid_constant__ CUtensorMap tm_e, const __grid_const
         inv_c[b][ct] = c < kept ? ms.kept_inv_norm[(size_t)bh * a.kept_stride + c] : 0.f;
       }
       merge_consumer_sync();
-      ok = __all_sync(0xffffffffu, merge_wait(&bars->acc_full[b], (t >> 1) & 1, bars, a.status, 45));
-      if (!ok) break;
+      // a warp whose wait gave up keeps walking the loop, so that it still meets the other consumers
+      // on the named barrier above; it only stops touching the accumulators
+      if (ok) ok = __all_sync(0xffffffffu, merge_wait(&bars->acc_full[b], (t >> 1) & 1, bars, a.status, 45, a.wait_cycles));
+      if (!ok) continue;
       tc_fence_after();
       const int n_valid = min(kTileM, kept - t * kTileM);
 #pragma unroll
@@ -490,14 +491,14 @@ int launch_merge_finish(const StepArgs& a, const MergeScratch& ms, cudaStream_t 
   constexpr int kRowsPerCta = (kApplyThreads / 32) * kApplyRowsPerWarp;
   const dim3 g_apply((kept + kRowsPerCta - 1) / kRowsPerCta, bh);
   if (a.head_dim == 128) {
-    allow_dynamic_smem(merge_assign_kernel<128>, assign_smem_bytes<128>());
+    if (!allow_dynamic_smem(merge_assign_kernel<128>, assign_smem_bytes<128>())) return -1;
     launch_k(merge_assign_kernel<128>, g_assign, kAssignThreads, assign_smem_bytes<128>(), st, te, tk, a, ms);
-    allow_dynamic_smem(merge_apply_kernel<128>, apply_smem_bytes<128>());
+    if (!allow_dynamic_smem(merge_apply_kernel<128>, apply_smem_bytes<128>())) return -1;
     launch_k(merge_apply_kernel<128>, g_apply, kApplyThreads, apply_smem_bytes<128>(), st, a, ms);
   } else {
-    allow_dynamic_smem(merge_assign_kernel<64>, assign_smem_bytes<64>());
+    if (!allow_dynamic_smem(merge_assign_kernel<64>, assign_smem_bytes<64>())) return -1;
     launch_k(merge_assign_kernel<64>, g_assign, kAssignThreads, assign_smem_bytes<64>(), st, te, tk, a, ms);
-    allow_dynamic_smem(merge_apply_kernel<64>, apply_smem_bytes<64>());
+    if (!allow_dynamic_smem(merge_apply_kernel<64>, apply_smem_bytes<64>())) return -1;
     launch_k(merge_apply_kernel<64>, g_apply, kApplyThreads, apply_smem_bytes<64>(), st, a, ms);
   }
   return launched(2);

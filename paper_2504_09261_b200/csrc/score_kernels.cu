@@ -182,7 +182,7 @@ int launch_score_t(const StepArgs& a, const void* q, const void* k_new, float* s
   constexpr int VEC = Elem<T>::kPerVec;
   const size_t smem = (size_t)kMaxObs * D * 4 +
                       (size_t)kScoreChunk * (D / VEC + 1) * 16;   // >= 32*128*4 for the logit tile
-  allow_dynamic_smem(score_logits_kernel<T, D>, smem);
+  if (!allow_dynamic_smem(score_logits_kernel<T, D>, smem)) return -1;
   dim3 g1((max_cand + kScoreChunk - 1) / kScoreChunk, bh);
   launch_k(score_logits_kernel<T, D>, g1, kScoreChunk, smem, st, 
       a, static_cast<const T*>(q), static_cast<const T*>(k_new), s.logits, s.partials, s.max_chunks);

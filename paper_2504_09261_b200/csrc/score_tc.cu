@@ -37,7 +37,6 @@ using namespace ptx;
 constexpr int kChunkTc = 128;
 constexpr int kScoreThreads = 192;
 constexpr int kAccBufs = 4;
-constexpr long long kScoreWaitCycles = 2000000000ll;   // about one second
 constexpr uint32_t kDrainSpins = 1u << 22;
 
 struct ScoreBars {
@@ -48,14 +47,14 @@ struct ScoreBars {
   int abort_flag;
 };
 
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, ScoreBars* b, int* status, int code) {
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, ScoreBars* b, int* status, int code, long long limit) {
   const uint32_t addr = smem_u32(bar);
   const long long t0 = clock64();
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(addr, parity)) return true;
     if ((it & 63u) == 63u) {
       if (*reinterpret_cast<volatile int*>(&b->abort_flag)) return false;
-      if (clock64() - t0 > kScoreWaitCycles) break;
+      if (clock64() - t0 > limit) break;
     }
   }
   *reinterpret_cast<volatile int*>(&b->abort_flag) = 1;
@@ -64,6 +63,13 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, ScoreBa
 }
 
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// All 128 consumers meet; true when `ok` holds for every one of them.
+__device__ __forceinline__ bool consumer_all(bool ok) {
+  uint32_t r;
+  asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(r) : "r"((uint32_t)ok) : "memory");
+  return r != 0;
+}
 
 template <int D, int MODE>
 __global__ void __launch_bounds__(kScoreThreads)
@@ -158,7 +164,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_const
       bool ok = true;
       for (int i = 0; i < n_run; ++i) {
         const int s = i % STAGES;
-        ok = wait_bar(&bars->empty[s], ((i / STAGES) & 1) ^ 1, bars, a.status, 11);
+        ok = wait_bar(&bars->empty[s], ((i / STAGES) & 1) ^ 1, bars, a.status, 11, a.wait_cycles);
         if (!ok) break;
         const int chunk = c_begin + i;
         const bool from_cache = chunk < n_sc;
@@ -186,8 +192,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_const
       bool ok = true;
       for (int i = 0; i < n_run && ok; ++i) {
         const int s = i % STAGES, b = i % kAccBufs;
-        ok = wait_bar(&bars->full[s], (i / STAGES) & 1, bars, a.status, 12);
-        if (ok) ok = wait_bar(&bars->acc_free[b], ((i / kAccBufs) & 1) ^ 1, bars, a.status, 13);
+        ok = wait_bar(&bars->full[s], (i / STAGES) & 1, bars, a.status, 12, a.wait_cycles);
+        if (ok) ok = wait_bar(&bars->acc_free[b], ((i / kAccBufs) & 1) ^ 1, bars, a.status, 13, a.wait_cycles);
         if (!ok) break;
         tc_fence_after();
         const uint64_t k_desc = smem_desc_sw128(k_sm + s * K_BYTES, 16, 1024);
@@ -234,7 +240,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_const
     bool ok = true;
     for (int i = 0; i < n_run; ++i) {
       const int b = i % kAccBufs;
-      ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full[b], (i / kAccBufs) & 1, bars, a.status, 14));
+      ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full[b], (i / kAccBufs) & 1, bars, a.status, 14, a.wait_cycles));
       if (!ok) break;
       tc_fence_after();
       uint32_t acc[kMaxObs];
@@ -266,7 +272,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_const
         }
       }
     }
-    if (MODE == 1 && ok) {
+    // one warp's wait may have given up while another's completed: the fold below meets on the
+    // consumers' named barrier, so all 128 consumers take the same branch
+    const bool all_ok = MODE == 1 ? consumer_all(ok) : ok;
+    if (MODE == 1 && all_ok) {
       // fold the 128 per-thread statistics of every row into one partial for this CTA; the last
       // accumulator has been read, so every MMA is complete and the ring can be reused
 #pragma unroll
@@ -317,14 +326,18 @@ int launch_t(const StepArgs& a, const CUtensorMap& tm_cache, const CUtensorMap& 
       total += (long long)c * heads / 2;             // the split between the types is not known here
     }
   // about two CTAs per SM over the whole grid, each with a run long enough to fill its pipeline
-  int per_cta = (int)((total + 2 * 148 - 1) / (2 * 148));
+  const int two_per_sm = 2 * sm_count();
+  int per_cta = (int)((total + two_per_sm - 1) / two_per_sm);
   per_cta = std::max(per_cta, 2);
   const int splits = (max_chunks + per_cta - 1) / per_cta;
-  if (splits > s.max_chunks) return -1;
+  if (splits > s.max_chunks) {
+    set_error("scoring: more CTAs per head than the partial-statistics scratch holds");
+    return -1;
+  }
   const size_t smem = 1024 + (size_t)STAGES * (D / 64) * kChunkTc * 128 + (size_t)(D / 64) * kMaxObs * 128 +
                       sizeof(ScoreBars) + 16;
-  allow_dynamic_smem(score_tc_kernel<D, 1>, smem);
-  allow_dynamic_smem(score_tc_kernel<D, 2>, smem);
+  if (!allow_dynamic_smem(score_tc_kernel<D, 1>, smem)) return -1;
+  if (!allow_dynamic_smem(score_tc_kernel<D, 2>, smem)) return -1;
   const dim3 grid(splits, heads);
   const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q);
   launch_k(score_tc_kernel<D, 1>, grid, kScoreThreads, smem, st, tm_cache, tm_new, a, qp, s.partials, s.max_chunks, per_cta, scores);
@@ -337,7 +350,10 @@ int launch_t(const StepArgs& a, const CUtensorMap& tm_cache, const CUtensorMap& 
 int launch_score_tc(const StepArgs& a, const void* q, const void* k_new, float* scores, const Scratch& s,
                     cudaStream_t st) {
   CUtensorMap tm_new;
-  if (!make_rows_map(&tm_new, k_new, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) return -1;
+  if (!make_rows_map(&tm_new, k_new, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) {
+    set_error("scoring: cuTensorMapEncodeTiled failed for the new scale's keys");
+    return -1;
+  }
   const CUtensorMap& tm_cache = *static_cast<const CUtensorMap*>(a.k_map);
   return a.head_dim == 128 ? launch_t<128>(a, tm_cache, tm_new, q, scores, s, st)
                            : launch_t<64>(a, tm_cache, tm_new, q, scores, s, st);

@@ -9,6 +9,9 @@ Feeding the GPU's scores to the oracle's selection keeps near-ties from cascadin
 cache contents; the selection itself is still decided by the oracle's own code.
 With fused=True a second cache is driven through hack_scale_step on the same inputs; its stored
 positions must equal the staged path's and its outputs must meet (iv) as well.
+With free_running=True a second oracle decides every selection from its own fp64 scores (no teacher
+forcing); the Jaccard overlap of its stored positions with the GPU's is recorded per step.  It is
+information, not a pass criterion: one near-tie decided the other way changes all later steps.
 """
 from __future__ import annotations
 
@@ -34,13 +37,16 @@ class ParityReport:
     max_score_err: float = 0.0          # max of |d| / (max(|s|,|s^|) + atol/rtol)
     max_out_abs: float = 0.0
     max_out_abs_fused: float = 0.0
+    jaccard: List[float] = field(default_factory=list)   # free-running oracle vs GPU, per compressed (step, head)
     problems: List[str] = field(default_factory=list)
 
     def summary(self) -> str:
         return (f"{self.workload}: steps={self.steps} heads={self.heads_checked} "
                 f"compressed={self.compressed_heads} score_err={self.max_score_err:.2e} "
                 f"out_abs={self.max_out_abs:.2e} fused_out_abs={self.max_out_abs_fused:.2e} "
-                f"problems={len(self.problems)}")
+                + (f"jaccard(min/mean)={min(self.jaccard):.4f}/{sum(self.jaccard) / len(self.jaccard):.4f} "
+                   if self.jaccard else "")
+                + f"problems={len(self.problems)}")
 
     def ok(self) -> bool:
         return not self.problems
@@ -83,23 +89,38 @@ def run_parity(cfg: WorkloadConfig, layers: Sequence[int], fused: bool = False,
                heads_per_layer: Optional[int] = None, policy: int = 0,
                budget_c: Optional[int] = None, budget_s: Optional[int] = None,
                scales: Optional[int] = None, check_rows: bool = True,
-               obs_sampler: int = 0, obs_rows=None) -> ParityReport:
+               obs_sampler: int = 0, obs_rows=None, pairs_of=None, gen_on_gpu: bool = False,
+               free_running: bool = False, staged_cache=None) -> ParityReport:
+    """pairs_of: {layer: [(b, h), ...]} overrides the per-layer sample; gen_on_gpu: the seeded
+    generator runs on the device and the oracle reads a host copy of the same bytes (the large
+    workloads would spend minutes in the CPU generator otherwise); staged_cache: a cache of the
+    same configuration to run the staged calls on (it is reset first and left open)."""
     dev = torch.device("cuda:0")
     tdt = _torch_dtype(cfg)
-    gen = SyntheticQKV(cfg)
+    gen = SyntheticQKV(cfg, device=dev if gen_on_gpu else "cpu")
     mask = gen.head_is_contextual.numpy()
     b_c = cfg.budget_c if budget_c is None else budget_c
     b_s = cfg.budget_s if budget_s is None else budget_s
     orc = ho.HackOracle(cfg.n_layers, cfg.n_heads, cfg.batch, cfg.head_dim, cfg.sides, mask, b_c, b_s,
                         n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, overflow_policy=policy,
                         obs_sampler=obs_sampler, obs_rows=obs_rows)
-    staged = make_cache(cfg, mask, policy, b_c, b_s, obs_sampler=obs_sampler, obs_rows=obs_rows)
+    if staged_cache is not None:
+        staged = staged_cache
+        staged.hack_reset()
+    else:
+        staged = make_cache(cfg, mask, policy, b_c, b_s, obs_sampler=obs_sampler, obs_rows=obs_rows)
     twin = make_cache(cfg, mask, policy, b_c, b_s, obs_sampler=obs_sampler, obs_rows=obs_rows) if fused else None
     rep = ParityReport(cfg.name)
     bh = cfg.batch * cfg.n_heads
     H = cfg.n_heads
     n_scales = cfg.n_scales if scales is None else scales
-    pairs_of = {l: sample_heads(cfg, l, heads_per_layer) for l in layers}
+    if pairs_of is None:
+        pairs_of = {l: sample_heads(cfg, l, heads_per_layer) for l in layers}
+    free = None
+    if free_running:
+        free = ho.HackOracle(cfg.n_layers, cfg.n_heads, cfg.batch, cfg.head_dim, cfg.sides, mask, b_c, b_s,
+                             n_obs=cfg.n_obs, n_init_scales=cfg.n_init_scales, overflow_policy=policy,
+                             obs_sampler=obs_sampler, obs_rows=obs_rows)
     out_tol = OUT_TOL[cfg.dtype]
     scores = torch.empty((bh, staged.cand_stride), dtype=torch.float32, device=dev)
     idx = torch.empty((bh, staged.kept_stride), dtype=torch.int32, device=dev)
@@ -113,6 +134,7 @@ def run_parity(cfg: WorkloadConfig, layers: Sequence[int], fused: bool = False,
         for l in layers:
             q, kk, v = gen.qkv(l, k)
             qd, kd, vd = q.to(dev), kk.to(dev), v.to(dev)
+            q, kk, v = q.cpu(), kk.cpu(), v.cpu()
             out = torch.full_like(qd, float("nan"))
             info = staged.hack_step_info(l, k)
             scores.fill_(float("nan"))
@@ -130,7 +152,6 @@ def run_parity(cfg: WorkloadConfig, layers: Sequence[int], fused: bool = False,
             s_h = scores.cpu().numpy()
             idx_h = idx.cpu().numpy()
             kept_h = kept.cpu().numpy()
-            out_h = out.to(torch.float64).cpu().numpy()
             pairs = pairs_of[l]
             override = {}
             for (b, h) in pairs:
@@ -139,8 +160,16 @@ def run_parity(cfg: WorkloadConfig, layers: Sequence[int], fused: bool = False,
                 cand = info.cand_c if ctx else info.cand_s
                 if trig:
                     override[(b, h)] = s_h[b * H + h, :cand].astype(np.float64)
-            o_ref, recs = orc.scale_step(l, k, q.to(torch.float64).numpy(), kk.to(torch.float64).numpy(),
-                                         v.to(torch.float64).numpy(), scores_override=override, heads=pairs)
+            if 2 * len(pairs) < bh:
+                # only the sampled heads are widened (the rest of the arrays is never read)
+                q64, k64, v64 = (np.zeros(tuple(t.shape)) for t in (q, kk, v))
+                for (b, h) in pairs:
+                    q64[b, h], k64[b, h], v64[b, h] = (t[b, h].to(torch.float64).numpy() for t in (q, kk, v))
+            else:
+                q64, k64, v64 = (t.to(torch.float64).numpy() for t in (q, kk, v))
+            o_ref, recs = orc.scale_step(l, k, q64, k64, v64, scores_override=override, heads=pairs)
+            if free is not None:
+                free.scale_step(l, k, q64, k64, v64, heads=pairs, need_output=False)
             lengths = staged.hack_get_lengths(l)
             for (b, h) in pairs:
                 tag = f"layer {l} scale {k} b {b} h {h}"
@@ -176,6 +205,10 @@ def run_parity(cfg: WorkloadConfig, layers: Sequence[int], fused: bool = False,
                     pos_g = np.frombuffer(staged.hack_read_head(l, b, h, 2), dtype=np.int32)
                     if not np.array_equal(pos_g.astype(np.int64), st.pos):
                         note(f"{tag}: stored positions differ")
+                    if free is not None and trig:
+                        pf = free.state[l][b][h].pos
+                        inter = np.intersect1d(pos_g.astype(np.int64), pf).shape[0]
+                        rep.jaccard.append(inter / max(pos_g.shape[0] + pf.shape[0] - inter, 1))
                     if staged.hack_read_head(l, b, h, 0) != _rows_bytes(st.k, tdt):
                         note(f"{tag}: stored K rows are not byte-equal")
                     if staged.hack_read_head(l, b, h, 1) != _rows_bytes(st.v, tdt):
@@ -184,7 +217,7 @@ def run_parity(cfg: WorkloadConfig, layers: Sequence[int], fused: bool = False,
                         pos_f = np.frombuffer(twin.hack_read_head(l, b, h, 2), dtype=np.int32)
                         if not np.array_equal(pos_f, pos_g):
                             note(f"{tag}: fused path kept a different set")
-                d = float(np.max(np.abs(out_h[b, h] - o_ref[b, h])))
+                d = float(np.max(np.abs(out[b, h].to(torch.float64).cpu().numpy() - o_ref[b, h])))
                 if not np.isfinite(d):
                     d = float("inf")
                 rep.max_out_abs = max(rep.max_out_abs, d)
@@ -198,7 +231,8 @@ def run_parity(cfg: WorkloadConfig, layers: Sequence[int], fused: bool = False,
                     if df > out_tol:
                         note(f"{tag}: fused attention output off by {df:.3e} (tol {out_tol})")
             rep.steps += 1
-    staged.close()
+    if staged_cache is None:
+        staged.close()
     if twin is not None:
         twin.close()
     return rep

@@ -19,7 +19,9 @@
 //    threads, and as few softmax instructions as possible: scale / sum / max work runs on packed
 //    or 3-input instructions.
 //  * Exponentials are scarce (16 per clock and SM against 8192 tensor flops): kPolyOf8 of every
-//    8 pairs are evaluated with a cubic on the FMA pipe instead.
+//    8 pairs can be evaluated with a cubic on the FMA pipe instead.  Two of eight made the loop
+//    2.4 % faster, but a probability from the cubic can round to the other bf16 neighbour than
+//    the one the row-sum correction below assumes, which cost 5e-3 of output accuracy: off.
 // TMEM (512 columns): S0 [0,128)  S1 [128,256)  O0 [256,256+D)  O1 [256+D,256+2D); the bf16
 // probabilities P_t overwrite the first 64 columns of S_t and feed the second MMA straight from
 // TMEM.  K tiles are K-major operands, V tiles MN-major operands, both 128-byte swizzled as TMA
@@ -52,7 +54,7 @@ constexpr int kBN = 128;                 // cache rows per K/V tile
 constexpr int kThreadsTc = 384;
 constexpr int kMmaWarp = 0, kProducerWarp = 1;   // the issuer is the oldest warp of its scheduler
 constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // 2*128*224 + 128*56 = 384*168 registers
-constexpr int kPolyOf8 = 2;              // pairs out of 8 whose 2^x runs on the FMA pipe
+constexpr int kPolyOf8 = 0;              // pairs out of 8 whose 2^x runs on the FMA pipe
 constexpr int kKStages = 2;
 constexpr int kVStages = 2;
 constexpr uint32_t kSpinLimit = 1u << 22;          // polls while draining after an abort
@@ -494,7 +496,7 @@ bool make_rows_map(void* out_map, const void* base, uint64_t rows, int head_dim)
 
 int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
                      const void* q, void* out, float* row_stats, const void* k_new, const void* v_new,
-                     cudaStream_t st) {
+                     int n_heads_served, cudaStream_t st) {
   CUtensorMap tm_q;
   if (!make_rows_map(&tm_q, q, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) {
     set_error("attention: cuTensorMapEncodeTiled failed for the queries");
@@ -503,9 +505,12 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
   TcParams p;
   p.n_heads = a.n_heads;
   p.n_new = a.n_new;
-  // one query tile per CTA while that still fits one wave: twice the CTAs, no idle SMs
   const int n_tiles = (a.n_new + kBM - 1) / kBM;
-  p.tiles_per_cta = n_tiles * a.batch * a.n_heads <= sm_count() ? 1 : 2;
+  // n_heads_served < all heads: only the first heads of head_order (those of one type) are served
+  const int heads = n_heads_served > 0 ? n_heads_served : a.batch * a.n_heads;
+  // one query tile per CTA while that still fits one wave: twice the CTAs, no idle SMs; a launch
+  // that serves one head type shares the GPU with the other type's kernels and keeps two
+  p.tiles_per_cta = (n_heads_served == 0 && n_tiles * heads <= sm_count()) ? 1 : 2;
   p.n_pairs = (n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
   const CUtensorMap& tk = *static_cast<const CUtensorMap*>(k_map);
   const CUtensorMap& tv = *static_cast<const CUtensorMap*>(v_map);
@@ -539,7 +544,7 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
   p.out = static_cast<__nv_bfloat16*>(out);
   p.row_stats = row_stats;
   p.status = a.status;
-  const int grid = p.n_pairs * a.batch * a.n_heads;
+  const int grid = p.n_pairs * heads;
   if (a.head_dim == 128) {
     if (!allow_dynamic_smem(attend_tc_kernel<128>, tc_smem_bytes<128>())) return -1;
     launch_k(attend_tc_kernel<128>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, tm_kn, tm_vn, p);

@@ -54,7 +54,7 @@ bool attend_tc_serves(const StepArgs& a, int dtype) {
 
 int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st) {
   if (attend_tc_serves(a, dtype))
-    return launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, nullptr, nullptr, st);
+    return launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, nullptr, nullptr, 0, st);
   return launch_attend_simt(a, dtype, q, out, st);
 }
 
@@ -115,6 +115,10 @@ struct hack_cache {
   size_t reserved_bytes = 0, peak_bytes = 0;
   uint64_t launches = 0;
   long long wait_cycles = hack::kDefaultWaitCycles;   // limit of the kernels' bounded waits
+  // fused step with one head type compressing: the attention of the other type runs beside the
+  // compression on this stream, forked from and joined to the caller's stream by the two events
+  cudaStream_t side_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool poisoned = false;                        // a launch failed after part of a step had been enqueued
   // optional per-stage device timing (score, select, compact, attend)
   bool timing = false;
@@ -499,6 +503,11 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
     HACK_TRY(cudaMemset(c->obs_rows, 0, (size_t)cfg->n_scales * hack::kMaxObs * sizeof(int32_t)));
     c->obs_rows_set.assign(cfg->n_scales, 0);
   }
+  if (cfg->dtype == HACK_BF16) {
+    HACK_TRY(cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking));
+    HACK_TRY(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
+    HACK_TRY(cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming));
+  }
   HACK_TRY(cudaMalloc(&c->status, sizeof(int)));
   HACK_TRY(cudaMemset(c->status, 0, sizeof(int)));
   HACK_TRY(cudaDeviceSynchronize());
@@ -532,6 +541,9 @@ hack_status_t hack_free_cache(hack_cache_t* c) {
     if (c->ev_step[sl]) cudaEventDestroy(c->ev_step[sl]);
     if (c->ev_out[sl]) cudaEventDestroy(c->ev_out[sl]);
   }
+  if (c->side_stream) cudaStreamDestroy(c->side_stream);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
   if (c->h2d_stream) cudaStreamDestroy(c->h2d_stream);
   if (c->d2h_stream) cudaStreamDestroy(c->d2h_stream);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
@@ -662,7 +674,7 @@ hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const 
 // from the caller's tensors and appended by the attention kernel itself.
 static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void* q, void* out, float* sigma,
                                  cudaStream_t st, const void* k_new = nullptr, const void* v_new = nullptr,
-                                 const int* seg_new = nullptr) {
+                                 const int* seg_new = nullptr, int only_type = -1, bool finish = true) {
   // lengths are already those after compaction
   LayerState& ls = c->layers[layer];
   hack_step_info_t p{};
@@ -678,21 +690,31 @@ static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void
     // Eq. 6 needs the statistics of every softmax row; the tensor-core attention kernel leaves them
     if (!hack::attend_tc_serves(a, c->cfg.dtype))
       return fail(HACK_ERR_UNSUPPORTED, "hack_attend_variance needs a bf16 cache and a scale of at least 32 tokens (128 query rows over all heads)");
-    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, c->attn_row_stats, nullptr, nullptr, st);
+    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, c->attn_row_stats, nullptr, nullptr, 0, st);
     if (n >= 0) {
       const int m = hack::launch_attention_variance(a, q, c->attn_row_stats, c->attn_block_var, c->var_blocks, sigma, st);
       n = m < 0 ? m : n + m;
     }
   } else if (seg_new) {
-    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, k_new, v_new, st);
+    int served = 0;
+    if (only_type >= 0) {
+      // the heads of one type: they lead the head order that puts that type first
+      const int bh = c->cfg.batch * c->cfg.n_heads;
+      const int n_ctx = c->cfg.batch * c->n_ctx_heads[layer];
+      served = only_type == 1 ? n_ctx : bh - n_ctx;
+      a.head_order = c->head_order + ((size_t)layer * 2 + only_type) * bh;
+    }
+    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, k_new, v_new, served, st);
   } else {
     n = hack::launch_attend(a, c->cfg.dtype, q, out, st);
   }
   if (n < 0) return HACK_ERR_CUDA;   // text recorded by the launcher
   ts.done(n);
   c->launches += n;
-  ls.phase = 0;
-  ls.next_scale = scale + 1;
+  if (finish) {
+    ls.phase = 0;
+    ls.next_scale = scale + 1;
+  }
   return HACK_OK;
 }
 
@@ -774,6 +796,19 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
     return HACK_OK;
   }
   bool compressed = false;
+  // One head type compresses, the other only appends: the attention of the appending heads does
+  // not depend on the compression, so it is enqueued on the cache's side stream, forked here (before
+  // the compression launch) and joined at the end of the step.  Every (batch, head) is independent,
+  // the two launches touch disjoint heads.
+  const int n_ctx_bh = c->cfg.batch * c->n_ctx_heads[layer];
+  const int n_heads_of[2] = {c->cfg.batch * c->cfg.n_heads - n_ctx_bh, n_ctx_bh};
+  const int trig_type = p.triggered_c ? 1 : 0;
+  const bool can_fork = any && fused_append && p.triggered_c != p.triggered_s && !c->timing && c->side_stream &&
+                        n_heads_of[0] > 0 && n_heads_of[1] > 0;
+  if (can_fork) {
+    HACK_CUDA(cudaEventRecord(c->ev_fork, st));
+    HACK_CUDA(cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0));
+  }
   if (any && fused_append) {
     // score, select and compact in one cluster launch per head (counted with the scoring stage)
     StageScope ts(c, st, 0);
@@ -781,6 +816,21 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
     ts.done(r);
     n += r;
     compressed = r > 0;
+  }
+  if (can_fork) {
+    if (compressed) {
+      c->launches += n;
+      advance_after_compact(c, layer, p);
+      s = attend_impl(c, layer, scale, q, out, nullptr, c->side_stream, k, v, seg_new, 1 - trig_type, false);
+      if (s == HACK_OK) s = attend_impl(c, layer, scale, q, out, nullptr, st, k, v, seg_new, trig_type, true);
+    }
+    // the side stream always comes back to the caller's stream (it may be part of a capture)
+    cudaEventRecord(c->ev_join, c->side_stream);
+    cudaStreamWaitEvent(st, c->ev_join, 0);
+    if (compressed) {
+      if (s == HACK_ERR_CUDA) c->poisoned = true;
+      return s;
+    }
   }
   if (any && !compressed) {
     {

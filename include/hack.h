@@ -261,6 +261,16 @@ HACK_API hack_status_t hack_poll_status(hack_cache_t* cache, void* stream);
  * (a limit of a few cycles makes the first wait that is not already satisfied give up) and for
  * callers that want a tighter bound than a second.  INVALID_ARG for a negative limit. */
 HACK_API hack_status_t hack_set_wait_limit(hack_cache_t* cache, int64_t cycles);
+/* 1 if this library is the checked build (compiled with HACK_DEBUG_CHECKS), else 0.  The checked
+ * build stands in for a memory checker: its kernels compare every ragged index they form with its
+ * bound, skip the access on a violation and put the site's code into the status word
+ * (hack_poll_status then returns HACK_ERR_STATE), and its planes carry one guard row behind the
+ * rows of every (layer, batch, head). */
+HACK_API int32_t hack_debug_build(void);
+/* Checked build only: synchronises the device and counts the guard rows (K, V and position planes)
+ * that no longer hold their pattern; hack_last_error() names the first.  UNSUPPORTED in the normal
+ * build. */
+HACK_API hack_status_t hack_debug_check(hack_cache_t* cache, int32_t* violations);
 /* Text of the calling thread's last error; never NULL. */
 HACK_API const char* hack_last_error(void);
 

@@ -10,7 +10,11 @@ import ctypes as C
 import os
 from typing import Optional, Sequence
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libhack_b200.so")
+# HACK_B200_CHECKED=1 selects the checked build of the same sources (bounds checks in the kernels,
+# guard rows in the planes); HackCache.close() then also verifies the guard rows.
+_CHECKED = os.environ.get("HACK_B200_CHECKED", "0") == "1"
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib",
+                         "libhack_b200_checked.so" if _CHECKED else "libhack_b200.so")
 
 HACK_OK, HACK_ERR_INVALID_ARG, HACK_ERR_UNSUPPORTED, HACK_ERR_OOM, HACK_ERR_CUDA, HACK_ERR_STATE, \
     HACK_ERR_TIMEOUT = range(7)
@@ -25,7 +29,7 @@ EXPORTS = (
     "hack_classify_heads", "hack_scale_step",
     "hack_scale_step_host", "hack_score_noalloc", "hack_get_lengths", "hack_read_head", "hack_kv_bytes",
     "hack_launch_count", "hack_stage_timing", "hack_stage_times", "hack_poll_status", "hack_set_wait_limit",
-    "hack_last_error",
+    "hack_debug_build", "hack_debug_check", "hack_last_error",
 )
 
 
@@ -88,6 +92,7 @@ def _load() -> C.CDLL:
         "hack_launch_count": [vp, C.POINTER(C.c_uint64)],
         "hack_poll_status": [vp, vp],
         "hack_set_wait_limit": [vp, C.c_int64],
+        "hack_debug_check": [vp, C.POINTER(i32)],
         "hack_stage_timing": [vp, i32],
         "hack_stage_times": [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint64)],
     }
@@ -95,6 +100,8 @@ def _load() -> C.CDLL:
         fn = getattr(lib, name)
         fn.argtypes = args
         fn.restype = C.c_int
+    lib.hack_debug_build.argtypes = []
+    lib.hack_debug_build.restype = C.c_int32
     return lib
 
 
@@ -171,8 +178,23 @@ class HackCache:
 
     def close(self) -> None:
         if getattr(self, "_h", None) is not None and self._h.value:
+            problem = None
+            if lib.hack_debug_build():
+                # checked build: no kernel may have tripped a bounds check or touched a guard row
+                if lib.hack_poll_status(self._h, None) != HACK_OK:
+                    problem = hack_last_error()
+                bad = C.c_int32()
+                if lib.hack_debug_check(self._h, C.byref(bad)) == HACK_OK and bad.value and problem is None:
+                    problem = f"{bad.value} guard rows overwritten: {hack_last_error()}"
             lib.hack_free_cache(self._h)
             self._h = C.c_void_p()
+            if problem:
+                raise HackError(HACK_ERR_STATE, problem)
+
+    def hack_debug_check(self) -> int:
+        bad = C.c_int32()
+        _check(lib.hack_debug_check(self._h, C.byref(bad)))
+        return bad.value
 
     def __del__(self):
         try:

@@ -152,7 +152,7 @@ append_attend_small_kernel(const StepArgs a, const T* __restrict__ q, const T* _
   // append: rows [stored, stored + n_new) of the cache take the new scale's rows; the CTAs of a
   // head share them, 16 bytes per thread
   constexpr int ROWV = D / VEC;                 // 16-byte pieces per row
-  const int n_pieces = a.n_new * ROWV;
+  const int n_pieces = dbg_ok(stored + a.n_new <= a.cap[ctx], a.status, 6) ? a.n_new * ROWV : 0;
   const uint4* ksrc = reinterpret_cast<const uint4*>(kn);
   const uint4* vsrc = reinterpret_cast<const uint4*>(vn);
   uint4* kdst = reinterpret_cast<uint4*>(static_cast<T*>(a.k_plane) + (off + stored) * D);
@@ -161,7 +161,7 @@ append_attend_small_kernel(const StepArgs a, const T* __restrict__ q, const T* _
     kdst[i] = ksrc[i];
     vdst[i] = vsrc[i];
   }
-  if (blockIdx.x == 0)
+  if (blockIdx.x == 0 && n_pieces > 0)
     for (int r = threadIdx.x; r < a.n_new; r += blockDim.x) a.pos_plane[off + stored + r] = a.pos_base + r;
 }
 

@@ -67,6 +67,7 @@ struct TcParams {
   int append_new;                        // heads with len_b > 0 also store those rows behind their len_a cache rows
   int pos_base;                          // global position of the new scale's first token
   int head_dim_pieces;                   // 16-byte pieces per row
+  int cap[2];                            // rows a head of each type owns (checked builds)
   long long wait_cycles;                 // limit of every mbarrier wait
   uint4* k_plane;                        // cache planes of this layer (append only)
   uint4* v_plane;
@@ -193,7 +194,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   if (warp == 2 || warp == 3) {
     reg_dec<kOtherRegs>();
-    if (p.append_new && len_b > 0) {
+    if (p.append_new && len_b > 0 && dbg_ok(len_a >= 0 && len_a + len_b <= p.cap[type], p.status, 7)) {
       // Eq. 3 for this head: the new scale's rows go behind the len_a cache rows.  The CTAs of the
       // head share the rows; whole rows of K and V, 16 bytes per thread, four loads in flight.
       const int per_cta = (len_b + p.n_pairs - 1) / p.n_pairs;
@@ -531,6 +532,8 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
   }
   p.pos_base = a.pos_base;
   p.head_dim_pieces = a.head_dim * 2 / 16;
+  p.cap[0] = a.cap[0];
+  p.cap[1] = a.cap[1];
   p.wait_cycles = a.wait_cycles;
   p.k_plane = static_cast<uint4*>(a.k_plane);
   p.v_plane = static_cast<uint4*>(a.v_plane);

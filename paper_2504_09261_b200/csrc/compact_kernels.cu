@@ -73,7 +73,10 @@ compact_move_kernel(const StepArgs a, const int32_t* __restrict__ idx, int row_p
       mv[u] = false;
       if (r < n_old) {
         const int src = list[r];
-        if (src != r) { val[u] = plane[(size_t)src * row_pieces + piece]; mv[u] = true; }
+        if (src != r && dbg_ok(src > r && src < stored && r < a.cap[ctx], a.status, 1)) {
+          val[u] = plane[(size_t)src * row_pieces + piece];
+          mv[u] = true;
+        }
       }
     }
     __syncthreads();
@@ -93,7 +96,7 @@ compact_move_kernel(const StepArgs a, const int32_t* __restrict__ idx, int row_p
         mv[u] = false;
         if (r < n_old) {
           const int src = list[r];
-          if (src != r) { val[u] = pos[src]; mv[u] = true; }
+          if (src != r && dbg_ok(src > r && src < stored, a.status, 2)) { val[u] = pos[src]; mv[u] = true; }
         }
       }
       __syncthreads();
@@ -126,11 +129,15 @@ compact_copy_kernel(const StepArgs a, const int32_t* __restrict__ idx, const uin
   for (int c0 = n_old + blockIdx.x * rows_per_pass * kCopyUnroll; c0 < n_keep;
        c0 += gridDim.x * rows_per_pass * kCopyUnroll) {
     uint4 val[kCopyUnroll];
+    bool ok[kCopyUnroll];
 #pragma unroll
     for (int u = 0; u < kCopyUnroll; ++u) {
       const int r = c0 + u * rows_per_pass + rsub;
+      ok[u] = false;
       if (r < n_keep) {
         const int src = (list ? list[r] : r) - stored;
+        ok[u] = dbg_ok(src >= 0 && src < a.n_new && r < a.cap[ctx], a.status, 3);
+        if (!ok[u]) continue;
         val[u] = fresh[(size_t)src * row_pieces + piece];
         if (plane_id == 0 && piece == 0) pos[r] = a.pos_base + src;
       }
@@ -138,7 +145,7 @@ compact_copy_kernel(const StepArgs a, const int32_t* __restrict__ idx, const uin
 #pragma unroll
     for (int u = 0; u < kCopyUnroll; ++u) {
       const int r = c0 + u * rows_per_pass + rsub;
-      if (r < n_keep) plane[(size_t)r * row_pieces + piece] = val[u];
+      if (r < n_keep && ok[u]) plane[(size_t)r * row_pieces + piece] = val[u];
     }
   }
 }

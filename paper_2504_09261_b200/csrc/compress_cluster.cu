@@ -473,7 +473,7 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
       const bool live = slot_info(i * kCkChunk + key_row, j);
       uint32_t key = 0;
       if (live) {
-        if (p.scores) p.scores[(size_t)bh * a.cand_stride + j] = s;
+        if (p.scores && dbg_ok(j < a.cand_stride, a.status, 8)) p.scores[(size_t)bh * a.cand_stride + j] = s;
         if (structural && (j < a.t_init || (a.protect_new && j >= stored))) {
           key = 0xffffffffu;
         } else {
@@ -585,10 +585,12 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
       if (slot < n_slots && slot_info(slot, j)) {
         const uint32_t k = keys[slot];
         if (k > thr) {
-          if (!(attend_appends && j >= stored)) list[gt_before + min(eq_before, need)] = j;
+          const int o = gt_before + min(eq_before, need);
+          if (!(attend_appends && j >= stored) && dbg_ok(o >= 0 && o < n_keep, a.status, 9)) list[o] = j;
           ++gt_before;
         } else if (k == thr) {
-          if (eq_before < need && !(attend_appends && j >= stored)) list[gt_before + eq_before] = j;
+          if (eq_before < need && !(attend_appends && j >= stored) && dbg_ok(gt_before + eq_before < n_keep, a.status, 9))
+            list[gt_before + eq_before] = j;
           ++eq_before;
         }
       }
@@ -616,7 +618,9 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
       const int first = r0 + rank * S;
       const int rows = max(0, min(S, n_rows - first));
       for (int lr = tid; lr < rows; lr += kCkThreads) {
-        const int src = list[first + lr];
+        int src = list[first + lr];
+        // a checked build turns an entry outside [dst, candidates) into "stays where it is"
+        if (!dbg_ok(src >= first + lr && src < stored + n_new && first + lr < a.cap[ctx], a.status, 10)) src = first + lr;
         src_stage[lr] = src;
         pos_stage[lr] = src < stored ? pos[src] : a.pos_base + (src - stored);
       }

@@ -70,6 +70,12 @@ struct LayerState {
 
 struct alignas(64) TensorMapBox { unsigned char bytes[128]; };
 
+#if defined(HACK_DEBUG_CHECKS)
+constexpr int kCanaryRows = 1;
+#else
+constexpr int kCanaryRows = 0;
+#endif
+
 struct hack_cache {
   hack_config_t cfg;
   std::vector<int32_t> sides, n_tok, t_cum;     // t_cum[k] = tokens of scales 0..k
@@ -185,6 +191,7 @@ hack::StepArgs make_args(const hack_cache* c, int layer, int scale, const hack_s
   a.stored[0] = p.stored_s; a.stored[1] = p.stored_c;
   a.cand[0] = p.cand_s;     a.cand[1] = p.cand_c;
   a.kept[0] = p.kept_s;     a.kept[1] = p.kept_c;
+  a.cap[0] = c->cap[0];     a.cap[1] = c->cap[1];
   a.trig[0] = p.triggered_s; a.trig[1] = p.triggered_c;
   a.n_obs_rows = p.n_obs_rows;
   // the query subset of Eq. 9: uniform spacing, or one of the ablation's alternatives
@@ -403,7 +410,7 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
       for (int h = 0; h < cfg->n_heads; ++h) {
         const int t = c->mask[(size_t)l * cfg->n_heads + h];
         row_off[(size_t)l * bh + b * cfg->n_heads + h] = (int32_t)rows;
-        rows += c->cap[t];
+        rows += c->cap[t] + kCanaryRows;            // checked builds: one guard row behind every head
         if (b == 0) n_ctx += t;
       }
     if (rows > (1ull << 30)) { delete c; return fail(HACK_ERR_UNSUPPORTED, "layer plane too large"); }
@@ -415,7 +422,7 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
   c->row_off_host = row_off;
   const size_t row_bytes = (size_t)cfg->head_dim * c->elt;
   const size_t pad_rows = 256;    // slack after the last layer so that tiled reads stay inside
-  c->reserved_bytes = 2 * total_rows * row_bytes;
+  c->reserved_bytes = 2 * (total_rows - (size_t)kCanaryRows * cfg->n_layers * bh) * row_bytes;   // K and V rows proper
 
   auto bail = [&](hack_status_t s) { hack_free_cache(c); return s; };
 #define HACK_TRY(call)                                                    \
@@ -432,6 +439,17 @@ hack_status_t hack_init_cache(const hack_config_t* cfg, hack_cache_t** out) {
   HACK_TRY(cudaMemset(c->k_all, 0, (total_rows + pad_rows) * row_bytes));
   HACK_TRY(cudaMemset(c->v_all, 0, (total_rows + pad_rows) * row_bytes));
   HACK_TRY(cudaMemset(c->pos_all, 0, (total_rows + pad_rows) * sizeof(int32_t)));
+  if (kCanaryRows) {
+    // guard rows carry a byte pattern no kernel writes; hack_debug_check looks for it later
+    for (int l = 0; l < cfg->n_layers; ++l)
+      for (int i = 0; i < bh; ++i) {
+        const int t = c->mask[(size_t)l * cfg->n_heads + i % cfg->n_heads];
+        const size_t row = c->layer_row_base[l] + row_off[(size_t)l * bh + i] + c->cap[t];
+        HACK_TRY(cudaMemset(c->k_all + row * row_bytes, hack::kCanaryByte, row_bytes));
+        HACK_TRY(cudaMemset(c->v_all + row * row_bytes, hack::kCanaryByte, row_bytes));
+        HACK_TRY(cudaMemset(c->pos_all + row, hack::kCanaryByte, sizeof(int32_t)));
+      }
+  }
   HACK_TRY(cudaMalloc(&c->row_off, row_off.size() * sizeof(int32_t)));
   HACK_TRY(cudaMemcpy(c->row_off, row_off.data(), row_off.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
   HACK_TRY(cudaMalloc(&c->mask_dev, c->mask.size()));
@@ -1004,10 +1022,50 @@ hack_status_t hack_poll_status(hack_cache_t* c, void* stream) {
   HACK_CUDA(cudaMemcpy(&word, c->status, sizeof(int), cudaMemcpyDeviceToHost));
   if (word != 0) {
     HACK_CUDA(cudaMemset(c->status, 0, sizeof(int)));
+    if (word >= hack::kDebugCodeBase) {
+      set_error("checked build: bounds check " + std::to_string(word - hack::kDebugCodeBase) + " failed in a kernel (the access was skipped)");
+      return HACK_ERR_STATE;
+    }
     set_error("a bounded device-side wait expired (status word " + std::to_string(word) + ")");
     return HACK_ERR_TIMEOUT;
   }
   return HACK_OK;
 }
+
+hack_status_t hack_debug_check(hack_cache_t* c, int32_t* violations) {
+  if (!c || !violations) return fail(HACK_ERR_INVALID_ARG, "cache or violations is NULL");
+  *violations = 0;
+  if (!kCanaryRows) return fail(HACK_ERR_UNSUPPORTED, "this library was built without HACK_DEBUG_CHECKS");
+  HACK_ON_DEVICE(c);
+  HACK_CUDA(cudaDeviceSynchronize());
+  const int bh = c->cfg.batch * c->cfg.n_heads;
+  const size_t row_bytes = (size_t)c->cfg.head_dim * c->elt;
+  std::vector<unsigned char> row(row_bytes);
+  int bad = 0;
+  for (int l = 0; l < c->cfg.n_layers; ++l)
+    for (int i = 0; i < bh; ++i) {
+      const int t = c->mask[(size_t)l * c->cfg.n_heads + i % c->cfg.n_heads];
+      const size_t r = c->layer_row_base[l] + c->row_off_host[(size_t)l * bh + i] + c->cap[t];
+      for (int which = 0; which < 3; ++which) {
+        const size_t n = which == 2 ? sizeof(int32_t) : row_bytes;
+        const unsigned char* src = which == 0 ? c->k_all + r * row_bytes
+                                  : which == 1 ? c->v_all + r * row_bytes
+                                               : reinterpret_cast<const unsigned char*>(c->pos_all + r);
+        HACK_CUDA(cudaMemcpy(row.data(), src, n, cudaMemcpyDeviceToHost));
+        bool hit = false;
+        for (size_t x = 0; x < n; ++x) hit = hit || row[x] != hack::kCanaryByte;
+        if (hit) {
+          if (bad == 0)
+            set_error("canary row overwritten: layer " + std::to_string(l) + ", (batch, head) " + std::to_string(i) +
+                      (which == 0 ? ", K plane" : which == 1 ? ", V plane" : ", position plane"));
+          ++bad;
+        }
+      }
+    }
+  *violations = bad;
+  return HACK_OK;
+}
+
+int32_t hack_debug_build(void) { return kCanaryRows; }
 
 }  // extern "C"

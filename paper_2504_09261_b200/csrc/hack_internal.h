@@ -23,6 +23,7 @@ struct StepArgs {
   int stored[2];        // L before the step
   int cand[2];          // T' = L + N_k
   int kept[2];          // length after the step
+  int cap[2];           // rows a head of this type owns in the planes (checked builds compare against it)
   int trig[2];          // compression triggered for this type
   int seg_new[2];       // tensor-core attention reads this type's new rows from the caller's K/V and
                         // appends them itself (the type keeps the whole new scale in this step)
@@ -141,7 +142,23 @@ inline void launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
   cfg.numAttrs = 1;
   cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
+// Checked build (-DHACK_DEBUG_CHECKS), the stand-in for a memory checker: every ragged index a
+// kernel forms (a list entry, a row of a head, a candidate, a slot of the index list) is compared
+// with its bound before it is used; on a violation the access is skipped and the code of the site
+// goes to the status word (nothing traps), which hack_poll_status reports.  The planes of a checked
+// build also carry a canary row behind every head, verified on the host by hack_debug_check.  In
+// the normal build the test is constant-true and costs nothing.
+constexpr int kDebugCodeBase = 100;     // status codes of the bounds checks start here
+constexpr unsigned char kCanaryByte = 0x5A;
 #if defined(__CUDACC__)
+#if defined(HACK_DEBUG_CHECKS)
+__device__ __forceinline__ bool dbg_ok(bool cond, int* status, int code) {
+  if (!cond) atomicExch(status, kDebugCodeBase + code);
+  return cond;
+}
+#else
+__device__ __forceinline__ bool dbg_ok(bool, int*, int) { return true; }
+#endif
 // Query row that serves as observation row i (Eq. 9's subset Q~).
 __device__ __forceinline__ int obs_row(const StepArgs& a, int i) {
   return a.obs_rows ? a.obs_rows[i] : a.obs_first + (int)(((long long)i * a.obs_span) / a.n_obs_rows);

@@ -153,10 +153,11 @@ select_reg_kernel(const StepArgs a, const float* __restrict__ scores, int32_t* _
   for (int e = 0; e < E; ++e) {
     const bool in = j0 + e < cand;
     if (in && key[e] > thr) {
-      out[gt_before + min(eq_before, need)] = j0 + e;
+      const int o = gt_before + min(eq_before, need);
+      if (dbg_ok(o >= 0 && o < n_keep, a.status, 4)) out[o] = j0 + e;
       ++gt_before;
     } else if (in && key[e] == thr) {
-      if (eq_before < need) out[gt_before + eq_before] = j0 + e;
+      if (eq_before < need && dbg_ok(gt_before + eq_before < n_keep, a.status, 4)) out[gt_before + eq_before] = j0 + e;
       ++eq_before;
     }
   }
@@ -218,7 +219,7 @@ select_kernel(const StepArgs a, const float* __restrict__ scores, int32_t* __res
     const int gt_before = packed & 0xffff, eq_before = eq_base + (packed >> 16);
     // entries equal to the threshold are kept while their running rank is below `need`
     const int pos = out_base + gt_before + min(eq_before, need) - min(eq_base, need);
-    if (gt || (eq && eq_before < need)) out[pos] = j;
+    if ((gt || (eq && eq_before < need)) && dbg_ok(pos >= 0 && pos < n_keep, a.status, 5)) out[pos] = j;
     out_base += (total & 0xffff) + min(eq_base + (total >> 16), need) - min(eq_base, need);
     eq_base += total >> 16;
   }

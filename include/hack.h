@@ -195,7 +195,12 @@ HACK_API hack_status_t hack_classify_heads(const double* sigma, int32_t n_layers
 
 /* The whole step for one (layer, scale): score -> select -> compact -> attend; heads whose
  * candidate count does not exceed their budget skip scoring and selection and keep everything
- * (section "KV Cache Compression for VAR": compress whenever the length exceeds the budget). */
+ * (section "KV Cache Compression for VAR": compress whenever the length exceeds the budget).
+ * bf16 caches: at most two launches (one cluster launch that scores, selects and compacts, one
+ * attention launch that also appends the rows of heads which keep the whole new scale).  When one
+ * head type compresses and the other only appends, the appending heads' attention is enqueued on a
+ * stream of the cache's own, forked from `stream` at the start of the call and joined to it before
+ * the call returns, so `stream` still orders everything (also inside a stream capture). */
 HACK_API hack_status_t hack_scale_step(hack_cache_t* cache, int32_t layer, int32_t scale, const void* q,
                               const void* k, const void* v, void* out, void* stream);
 
@@ -211,8 +216,11 @@ HACK_API hack_status_t hack_scale_step(hack_cache_t* cache, int32_t layer, int32
  * Intermediates live in a fixed array inside the library's device image (about 8.3 MiB, held
  * by every GPU that loads the library until the process exits), hence the limits
  * n_rows <= 512 and n_rows*n_cand <= 65536; larger sizes return HACK_ERR_UNSUPPORTED.
- * No cudaMalloc, cudaFree or other allocating call is made.  The first call on a device resolves
- * the array's address (cudaGetSymbolAddress); make that first call before any stream capture.
+ * No cudaMalloc, cudaFree or other allocating call is made.  The first call on a device is a
+ * set-up call: it resolves the array's address (cudaGetSymbolAddress) and, because CUDA loads a
+ * module's device image lazily, it is also the moment the driver reserves those 8.3 MiB on that
+ * device.  Make it at start-up, before the caller's own pool claims the rest of the memory and
+ * before any stream capture; every later call on that device leaves the device's memory as it is.
  * All calls share the array: calls that overlap on the GPU race, so keep them on one stream or
  * order them yourself.  Only enqueues; does not synchronise. */
 HACK_API hack_status_t hack_score_noalloc(const void* q, const void* k_cand, float* scores,
@@ -248,7 +256,9 @@ HACK_API hack_status_t hack_launch_count(const hack_cache_t* cache, uint64_t* la
  * stage); accumulators are cleared.  Synchronises the device. */
 HACK_API hack_status_t hack_stage_timing(hack_cache_t* cache, int32_t enable);
 /* Synchronises the device and returns the accumulated device time in ms and the number of kernel
- * launches per stage since timing was enabled: [0] score, [1] select, [2] compact, [3] attend. */
+ * launches per stage since timing was enabled: [0] score, [1] select, [2] compact, [3] attend.  In
+ * hack_scale_step on a bf16 cache scoring, selection and compaction are one launch, counted under
+ * [0]; while timing is on, the step does not run the two head types' work side by side. */
 HACK_API hack_status_t hack_stage_times(hack_cache_t* cache, double* ms, uint64_t* launches);
 /* Synchronises `stream`, then reports the device status word: HACK_OK, or HACK_ERR_TIMEOUT if a
  * bounded device-side wait gave up (the word is cleared by the call). */

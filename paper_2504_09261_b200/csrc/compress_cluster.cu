@@ -55,7 +55,7 @@ constexpr int kMaxOver = 6;                // chunks per CTA whose logits live i
 constexpr int kMaxCpc = kTmemChunks - 1 + kMaxOver;      // 21 chunks = 2688 keys per CTA
 constexpr int kMaxCluster = 8;
 constexpr uint32_t kCkDrainSpins = 1u << 22;
-constexpr int kMaxStages = 8;              // key tiles in flight per CTA
+constexpr int kMaxStages = 4;              // key tiles in flight per CTA (deeper rings measured no faster)
 constexpr int kMaxStageRows = 512;         // rows one CTA stages per round of the compaction
 constexpr size_t kSmemBudget = 227 * 1024; // dynamic shared memory a CTA may ask for
 static_assert(kCkThreads == 256, "one thread per histogram bin");

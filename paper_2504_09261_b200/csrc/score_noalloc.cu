@@ -9,7 +9,9 @@
 // statistics in a fixed array that lives in the library's own device image.
 //
 // The array (kScratchFloats floats, about 8.3 MiB) is part of the module: every GPU that loads
-// the library holds it until the process exits.  All calls share it and it keeps the previous
+// the library holds it until the process exits.  CUDA loads the module's device image lazily, so
+// the driver reserves it on a device during the first call made there (the set-up call, to be made
+// at start-up); no later call changes the device's memory.  All calls share it and it keeps the previous
 // call's contents; nothing in it has to start at zero because pass 1 overwrites every element
 // pass 2 reads.  Two calls that overlap on the GPU (different streams, or different host threads
 // without ordering) race on it: serialise them.
@@ -180,9 +182,8 @@ cudaError_t run(const DenseArgs& a, int n_rows, const void* q, const void* k, fl
                 float* scores, int score_stride, cudaStream_t st) {
   constexpr int VEC = Ld<T>::kPerVec;
   const size_t smem = (size_t)kMaxObs * D * 4 + (size_t)kChunk * (D / VEC + 1) * 16;
-  cudaError_t e = cudaFuncSetAttribute(noalloc_logits_kernel<T, D>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
+  // opt-in to more than 48 KB of dynamic shared memory, once per (kernel, device)
+  if (!allow_dynamic_smem(noalloc_logits_kernel<T, D>, smem)) return cudaErrorInvalidValue;
   float* logits = scratch;
   float* partials = scratch + kLogitFloats;
   noalloc_logits_kernel<T, D><<<dim3(a.chunks_per_row, n_rows), kChunk, smem, st>>>(

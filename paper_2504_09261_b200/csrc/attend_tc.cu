@@ -4,12 +4,15 @@
 //
 // One CTA serves one (batch, head) and up to two 128-row query tiles, which take turns on the
 // tensor pipe so that the softmax of one tile overlaps the MMAs of the other.
-//   warp  0     : tcgen05.mma issuer; also owns the TMEM allocation
+//   warp  0     : issuer of the Q K^T products; also owns the TMEM allocation
 //   warp  1     : TMA producer (K and V tiles of 128 cache rows through rings)
+//   warp  2     : issuer of the P V products (a single issuing thread for both products was the
+//                 bottleneck of the CTA: 0.212 -> 0.174 ms on the largest launch)
+//   warp  3     : appends the new scale's rows to the cache with bulk copies (heads that keep it whole)
 //   warps 4-7   : softmax of tile 0 (thread r owns query row r: one TMEM lane, no shuffles)
 //   warps 8-11  : softmax of tile 1
-//   warps 2-3 only complete the first warpgroup, which hands most of its registers to the
-//   softmax warpgroups (setmaxnreg) so that a whole 128-column score row lives in registers.
+//   The first warpgroup hands most of its registers to the softmax warpgroups (setmaxnreg) so that
+//   a whole 128-column score row lives in registers.
 //
 // What shapes the kernel (all measured on the device):
 //  * The thread that issues the MMAs needs instruction-issue slots of its scheduler; many busy
@@ -22,21 +25,27 @@
 //    8 pairs can be evaluated with a cubic on the FMA pipe instead.  Two of eight made the loop
 //    2.4 % faster, but a probability from the cubic can round to the other bf16 neighbour than
 //    the one the row-sum correction below assumes, which cost 5e-3 of output accuracy: off.
-// TMEM (512 columns): S0 [0,128)  S1 [128,256)  O0 [256,256+D)  O1 [256+D,256+2D); the bf16
-// probabilities P_t overwrite the first 64 columns of S_t and feed the second MMA straight from
-// TMEM.  K tiles are K-major operands, V tiles MN-major operands, both 128-byte swizzled as TMA
+// TMEM (512 columns): S [0,128)  P0 [128,192)  P1 [192,256)  O0 [256,256+D)  O1 [256+D,256+2D).
+// There is ONE logit buffer, which the two tiles use in turn, and a probability buffer per tile.  A
+// softmax thread reads its whole logit row into registers first and hands the buffer back at once
+// (s_free), so the next Q K^T product (the other tile's, or with one tile per CTA this tile's next
+// block) runs while it computes; the probabilities go to the tile's own buffer, from where the
+// second MMA takes them, so that no product waits for another to release columns it writes.  With
+// one buffer per tile holding first the logits and then the probabilities (the earlier form), each
+// tile was a serial chain softmax -> P V -> Q K^T -> softmax of about 3 400 cycles per 128 keys,
+// and the two tiles only interleaved; now the tensor pipe and the exponentials each run at their own
+// rate.  K tiles are K-major operands, V tiles MN-major operands, both 128-byte swizzled as TMA
 // writes them.  Softmax keeps a running maximum that is only raised (and O rescaled in TMEM) when
 // a row's maximum grows by more than 2^32, so rescaling is rare after the first tile.
-// (Tried and dropped: logits in two buffers of 64 keys per tile, so that the next Q K^T product
-// runs under the softmax.  The 128 x 64 x 16 MMA re-reads the whole Q operand from shared memory
-// for half the keys and takes nearly as long as the 128 x 128 x 16 one: the last-scale launch of the
-// 10 521-token workload went from 0.233 to 0.301 ms.)
+// (Tried and dropped: logits in two buffers of 64 keys per tile.  The 128 x 64 x 16 MMA re-reads the
+// whole Q operand from shared memory for half the keys and takes nearly as long as the
+// 128 x 128 x 16 one: the last-scale launch of the 10 521-token workload went from 0.233 to 0.301 ms.)
 // The keys and values of a head come in two segments: len_a rows of the head's cache, then len_b
 // rows of the new scale taken straight from the caller's K/V tensors (second pair of tensor maps).
 // Heads that keep the whole new scale (steps without eviction; structural heads, whose latest scale
 // is protected, Eq. 11) are served that way before the new rows are in the cache: the append
-// (Eq. 3) is done by warps 2-3 of the same CTAs, global to global, each CTA of a head taking a
-// slice of the rows; nothing in this launch reads the rows they write.
+// (Eq. 3) is done by warp 3 of the same CTAs with bulk copies through a small staging buffer, each
+// CTA of a head taking a slice of the rows; nothing in this launch reads the rows they write.
 // Every mbarrier wait is bounded; on expiry the CTA raises the status word, drains what it has in
 // flight, frees its TMEM and returns.
 #include <cuda.h>
@@ -52,12 +61,13 @@ using namespace ptx;
 constexpr int kBM = 128;                 // query rows per tile
 constexpr int kBN = 128;                 // cache rows per K/V tile
 constexpr int kThreadsTc = 384;
-constexpr int kMmaWarp = 0, kProducerWarp = 1;   // the issuer is the oldest warp of its scheduler
+constexpr int kMmaWarp = 0, kProducerWarp = 1, kPvWarp = 2, kAppendWarp = 3;   // an issuer is the oldest warp of its scheduler
 constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // 2*128*224 + 128*56 = 384*168 registers
 constexpr int kPolyOf8 = 0;              // pairs out of 8 whose 2^x runs on the FMA pipe
 constexpr int kKStages = 2;
 constexpr int kVStages = 2;
 constexpr uint32_t kSpinLimit = 1u << 22;          // polls while draining after an abort
+constexpr uint32_t kCopyChunk = 16384;             // bytes per bulk copy of the append
 constexpr float kRescaleThreshold = 32.0f;   // log2 units: p <= 2^32, far inside the bf16 / fp32 range
 
 struct TcParams {
@@ -87,8 +97,9 @@ struct Bars {
   uint64_t q_full[2];
   uint64_t k_full[kKStages], k_empty[kKStages];
   uint64_t v_full[kVStages], v_empty[kVStages];
-  uint64_t s_full[2], p_full[2][2], o_final[2];    // p_full[t][half]: P of 64 keys is in TMEM
-  uint64_t drain;
+  uint64_t s_full[2], s_free, p_full[2], p_free[2], o_final[2];
+  uint64_t copy_full[2];                            // append: a chunk of new rows has landed in its staging half
+  uint64_t drain, drain2;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -118,7 +129,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   constexpr int SUB = D / 64;                       // 64-column (128-byte) sub-tiles per row
   constexpr uint32_t SUB_BYTES = kBN * 128;         // one sub-tile: 128 rows x 128 bytes
   constexpr uint32_t TILE_BYTES = SUB * SUB_BYTES;
-  constexpr uint32_t S_COL = 0, O_COL = 256;
+  constexpr uint32_t S_COL = 0, P_COL = 128, O_COL = 256;
 
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t raw = smem_u32(smem_dyn);
@@ -127,7 +138,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t q_sm = base;
   const uint32_t k_sm = q_sm + 2 * TILE_BYTES;
   const uint32_t v_sm = k_sm + kKStages * TILE_BYTES;
-  Bars* bars = reinterpret_cast<Bars*>(sm + (2 + kKStages + kVStages) * TILE_BYTES);
+  const uint32_t copy_sm = v_sm + kVStages * TILE_BYTES;           // 2 x kCopyChunk bytes: staging of the append
+  Bars* bars = reinterpret_cast<Bars*>(sm + (2 + kKStages + kVStages) * TILE_BYTES + 2 * kCopyChunk);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bh = p.head_order[blockIdx.x / p.n_pairs];
@@ -151,13 +163,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(&bars->q_full[t]), 1);
       mbar_init(smem_u32(&bars->s_full[t]), 1);
-      mbar_init(smem_u32(&bars->p_full[t][0]), 4);  // one arrival per warp of the tile
-      mbar_init(smem_u32(&bars->p_full[t][1]), 4);
+      mbar_init(smem_u32(&bars->p_full[t]), 4);     // one arrival per warp of the tile
+      mbar_init(smem_u32(&bars->p_free[t]), 1);
       mbar_init(smem_u32(&bars->o_final[t]), 1);
     }
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1); }
     for (int s = 0; s < kVStages; ++s) { mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1); }
+    mbar_init(smem_u32(&bars->s_free), 4);          // the four warps of the tile whose logits were in the buffer
+    mbar_init(smem_u32(&bars->copy_full[0]), 1);
+    mbar_init(smem_u32(&bars->copy_full[1]), 1);
     mbar_init(smem_u32(&bars->drain), 1);
+    mbar_init(smem_u32(&bars->drain2), 1);
     bars->abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
@@ -192,32 +208,70 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
   pdl_wait();     // everything above overlaps the tail of the previous kernel
 
-  if (warp == 2 || warp == 3) {
+  if (warp == kPvWarp) {
+    // ------------------------------------------------------------------ issuer of the P V products
+    // (a thread of its own: one thread issuing both products was the bottleneck of the CTA)
     reg_dec<kOtherRegs>();
-    if (p.append_new && len_b > 0 && dbg_ok(len_a >= 0 && len_a + len_b <= p.cap[type], p.status, 7)) {
-      // Eq. 3 for this head: the new scale's rows go behind the len_a cache rows.  The CTAs of the
-      // head share the rows; whole rows of K and V, 16 bytes per thread, four loads in flight.
-      const int per_cta = (len_b + p.n_pairs - 1) / p.n_pairs;
-      const int r0 = pair * per_cta, r1 = min(len_b, r0 + per_cta);
-      const int pieces = p.head_dim_pieces;
-      const int t = tid - 64;                                   // 0..63
-      const size_t src0 = (size_t)nrow * pieces, dst0 = (size_t)(krow + len_a) * pieces;
-      const int n = max(r1 - r0, 0) * pieces;
-      const int first = r0 * pieces;
-      for (int i0 = 0; i0 < n; i0 += 64 * 4) {
-        uint4 kv[4], vv[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int i = i0 + u * 64 + t;
-          if (i < n) { kv[u] = p.k_new[src0 + first + i]; vv[u] = p.v_new[src0 + first + i]; }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int i = i0 + u * 64 + t;
-          if (i < n) { p.k_plane[dst0 + first + i] = kv[u]; p.v_plane[dst0 + first + i] = vv[u]; }
+    if (lane == 0) {
+      constexpr uint32_t IDESC_PV = idesc_bf16_f32(kBM, D, 1);         // A = P (TMEM), B = V (MN-major)
+      const uint64_t v_desc0 = smem_desc_sw128(v_sm, SUB_BYTES, 1024);
+      bool ok = true;
+      for (int j = 0; j < nblk && ok; ++j) {
+        const int vs = j % kVStages;
+        const uint64_t vd = v_desc0 + (uint64_t)((vs * TILE_BYTES) >> 4);
+        for (int t = 0; t < ntile && ok; ++t) {
+          ok = wait_bar(&bars->p_full[t], j & 1, bars, p.status, 5, wlim);
+          if (ok && t == 0) ok = wait_bar(&bars->v_full[vs], (j / kVStages) & 1, bars, p.status, 6, wlim);
+          if (!ok) break;
+          tc_fence_after();
+          mma_ts_chain4(tmem + O_COL + t * D, tmem + P_COL + t * 64, vd, IDESC_PV, j > 0);
+          mma_ts_chain4(tmem + O_COL + t * D, tmem + P_COL + t * 64 + 32, vd + 4 * 128, IDESC_PV, 1);
+          mma_commit(smem_u32(&bars->p_free[t]));             // P_t may be rewritten, O_t is up to date
+          if (t == ntile - 1) mma_commit(smem_u32(&bars->v_empty[vs]));
+          if (j + 1 == nblk) mma_commit(smem_u32(&bars->o_final[t]));
         }
       }
-      for (int r = r0 + t; r < r1; r += 64) p.pos_plane[krow + len_a + r] = p.pos_base + r;
+      if (!ok) {
+        mma_commit(smem_u32(&bars->drain2));
+        const uint32_t bar = smem_u32(&bars->drain2);
+        for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar, 0); ++it) {}
+      }
+    }
+  } else if (warp == kAppendWarp) {
+    reg_dec<kOtherRegs>();
+    if (p.append_new && len_b > 0 && dbg_ok(len_a >= 0 && len_a + len_b <= p.cap[type], p.status, 7)) {
+      // Eq. 3 for this head: the new scale's rows go behind the len_a cache rows.  The rows are one
+      // contiguous run in the caller's tensor and in the cache plane; the CTAs of the head share
+      // them, and one thread moves this CTA's slice with bulk copies through two staging halves
+      // (global -> shared -> global), so the append costs no registers and no issue slots.
+      const int per_cta = (len_b + p.n_pairs - 1) / p.n_pairs;
+      const int r0 = pair * per_cta, r1 = min(len_b, r0 + per_cta);
+      for (int r = r0 + lane; r < r1; r += 32) p.pos_plane[krow + len_a + r] = p.pos_base + r;
+      if (lane == 0 && r1 > r0) {
+        const uint32_t row_bytes = (uint32_t)p.head_dim_pieces * 16;
+        const size_t src_off = ((size_t)nrow + r0) * row_bytes, dst_off = ((size_t)krow + len_a + r0) * row_bytes;
+        const uint32_t total = (uint32_t)(r1 - r0) * row_bytes;
+        const uint32_t n_chunks = (total + kCopyChunk - 1) / kCopyChunk;
+        bool ok = true;
+        uint32_t n = 0;                              // chunk counter over both planes
+        for (int plane = 0; plane < 2 && ok; ++plane) {
+          const unsigned char* src = reinterpret_cast<const unsigned char*>(plane == 0 ? p.k_new : p.v_new) + src_off;
+          unsigned char* dst = reinterpret_cast<unsigned char*>(plane == 0 ? p.k_plane : p.v_plane) + dst_off;
+          for (uint32_t ch = 0; ch < n_chunks && ok; ++ch, ++n) {
+            const uint32_t half = n & 1;
+            const uint32_t bytes = min(kCopyChunk, total - ch * kCopyChunk);
+            const uint32_t bar = smem_u32(&bars->copy_full[half]);
+            bulk_wait_read<1>();                     // the store that last read this half (two chunks ago) is done with it
+            mbar_expect_tx(bar, bytes);
+            bulk_load(copy_sm + half * kCopyChunk, src + (size_t)ch * kCopyChunk, bytes, bar);
+            ok = wait_bar(&bars->copy_full[half], (n >> 1) & 1, bars, p.status, 12, wlim);
+            if (!ok) break;
+            bulk_store(dst + (size_t)ch * kCopyChunk, copy_sm + half * kCopyChunk, bytes);
+            bulk_commit();
+          }
+        }
+        bulk_wait<0>();                              // every store has been performed before the CTA may leave
+      }
     }
   } else if (warp == kProducerWarp) {
     // ------------------------------------------------------------------ TMA producer
@@ -264,55 +318,43 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
   } else if (warp == kMmaWarp) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ issuer of the Q K^T products
     reg_dec<kOtherRegs>();
     if (lane == 0) {
       constexpr uint32_t IDESC_S = idesc_bf16_f32(kBM, kBN, 0);        // A = Q, B = K (both K-major)
-      constexpr uint32_t IDESC_PV = idesc_bf16_f32(kBM, D, 1);         // A = P (TMEM), B = V (MN-major)
       // descriptors of the tile bases; a k-step only adds a constant to the address field
       const uint64_t q_desc[2] = {smem_desc_sw128(q_sm, 16, 1024), smem_desc_sw128(q_sm + TILE_BYTES, 16, 1024)};
       const uint64_t k_desc0 = smem_desc_sw128(k_sm, 16, 1024);
-      const uint64_t v_desc0 = smem_desc_sw128(v_sm, SUB_BYTES, 1024);
       bool ok = true;
-      auto issue_s = [&](int t, int j) {
+      // S = Q_t K_j^T into the one logit buffer; `use` counts the products issued so far, and product
+      // number use needs the logits of product use - 1 to have left the buffer (s_free phase use - 1)
+      int use = 0;
+      auto issue_s = [&](int t, int j) -> bool {
+        if (use > 0 && !wait_bar(&bars->s_free, (use - 1) & 1, bars, p.status, 10, wlim)) return false;
+        tc_fence_after();
         const uint64_t kd = k_desc0 + (uint64_t)(((j % kKStages) * TILE_BYTES) >> 4);
-        if constexpr (D == 128) mma_ss_chain8(tmem + S_COL + t * kBN, q_desc[t], kd, IDESC_S, 0);
-        else mma_ss_chain4(tmem + S_COL + t * kBN, q_desc[t], kd, IDESC_S, 0);
+        if constexpr (D == 128) mma_ss_chain8(tmem + S_COL, q_desc[t], kd, IDESC_S, 0);
+        else mma_ss_chain4(tmem + S_COL, q_desc[t], kd, IDESC_S, 0);
         mma_commit(smem_u32(&bars->s_full[t]));
+        ++use;
+        return true;
       };
       for (int t = 0; t < ntile && ok; ++t) ok = wait_bar(&bars->q_full[t], 0, bars, p.status, 3, wlim);
       if (ok) ok = wait_bar(&bars->k_full[0], 0, bars, p.status, 4, wlim);
-      if (ok) {
-        tc_fence_after();
-        for (int t = 0; t < ntile; ++t) issue_s(t, 0);
-        mma_commit(smem_u32(&bars->k_empty[0]));
-      }
+      for (int t = 0; t < ntile && ok; ++t) ok = issue_s(t, 0);
+      if (ok) mma_commit(smem_u32(&bars->k_empty[0]));
       for (int j = 0; j < nblk && ok; ++j) {
-        const int vs = j % kVStages;
-        const uint64_t vd = v_desc0 + (uint64_t)((vs * TILE_BYTES) >> 4);
         for (int t = 0; t < ntile && ok; ++t) {
-          // the probabilities arrive in two halves of 64 keys, so that the second MMA starts while
-          // the softmax is still working on the second half
-          ok = wait_bar(&bars->p_full[t][0], j & 1, bars, p.status, 5, wlim);
-          if (ok && t == 0) ok = wait_bar(&bars->v_full[vs], (j / kVStages) & 1, bars, p.status, 6, wlim);
-          if (!ok) break;
-          tc_fence_after();
-          mma_ts_chain4(tmem + O_COL + t * D, tmem + S_COL + t * kBN, vd, IDESC_PV, j > 0);
-          ok = wait_bar(&bars->p_full[t][1], j & 1, bars, p.status, 5, wlim);
-          if (!ok) break;
-          tc_fence_after();
-          mma_ts_chain4(tmem + O_COL + t * D, tmem + S_COL + t * kBN + 32, vd + 4 * 128, IDESC_PV, 1);
-          if (t == ntile - 1) mma_commit(smem_u32(&bars->v_empty[vs]));
+          // the next logits of this tile: they only wait for the buffer, not for this tile's
+          // softmax, and so run under it
           if (j + 1 < nblk) {
             if (t == 0) {
               ok = wait_bar(&bars->k_full[(j + 1) % kKStages], ((j + 1) / kKStages) & 1, bars, p.status, 7, wlim);
               if (!ok) break;
-              tc_fence_after();
             }
-            issue_s(t, j + 1);
+            ok = issue_s(t, j + 1);
+            if (!ok) break;
             if (t == ntile - 1) mma_commit(smem_u32(&bars->k_empty[(j + 1) % kKStages]));
-          } else {
-            mma_commit(smem_u32(&bars->o_final[t]));
           }
         }
       }
@@ -329,7 +371,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     if (t < ntile) {
       const int r = tid & 127;                     // query row inside the tile == TMEM lane
       const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
-      const uint32_t s_addr = tmem + lane_addr + S_COL + t * kBN;
+      const uint32_t s_addr = tmem + lane_addr + S_COL;
+      const uint32_t p_addr = tmem + lane_addr + P_COL + t * 64;
       const uint32_t o_addr = tmem + lane_addr + O_COL + t * D;
       const float c = p.scale_log2;
       float m_used = -INFINITY, l = 0.f;
@@ -342,6 +385,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
         for (int ch = 0; ch < kBN / 32; ++ch) tmem_ld32(s_addr + ch * 32, sr + ch * 32);
         tmem_wait_ld();
+        // the logits are in registers: the buffer goes back to the MMA warp at once
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->s_free));
         // live keys of this tile: fewer than 128 only in the last tile of either segment
         const int valid = j < nblk_a ? len_a - j * kBN : len_b - (j - nblk_a) * kBN;
         if (valid < kBN) {
@@ -349,33 +396,32 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           for (int i = 0; i < kBN; ++i)
             if (i >= valid) sr[i] = 0xff800000u;   // -inf
         }
-        float mx4[4];
+        // row maximum, kept apart for the pairs whose exponential runs on the FMA pipe (pair index
+        // i with (i & 7) < kPolyOf8) and for the others: the row-sum correction below must form the
+        // largest probability with the same instructions the loop uses for that element
+        float mx_sfu[4], mx_fma[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          mx4[u] = fmaxf(__uint_as_float(sr[u * 32]), __uint_as_float(sr[u * 32 + 1]));
+          mx_sfu[u] = -INFINITY;
+          mx_fma[u] = -INFINITY;
 #pragma unroll
-          for (int i = 2; i < 32; i += 2)
-            mx4[u] = max3(mx4[u], __uint_as_float(sr[u * 32 + i]), __uint_as_float(sr[u * 32 + i + 1]));
+          for (int i = 0; i < 16; ++i) {
+            const float e0 = __uint_as_float(sr[u * 32 + 2 * i]), e1 = __uint_as_float(sr[u * 32 + 2 * i + 1]);
+            if ((i & 7) < kPolyOf8) mx_fma[u] = max3(mx_fma[u], e0, e1);
+            else mx_sfu[u] = max3(mx_sfu[u], e0, e1);
+          }
         }
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        const float mxs = fmaxf(fmaxf(mx_sfu[0], mx_sfu[1]), fmaxf(mx_sfu[2], mx_sfu[3]));
+        const float mxf = fmaxf(fmaxf(mx_fma[0], mx_fma[1]), fmaxf(mx_fma[2], mx_fma[3]));
+        const float mx = fmaxf(mxs, mxf);
         const bool grow = (mx - m_used) * c > kRescaleThreshold;     // always true in the first tile
-        if (__any_sync(0xffffffffu, grow)) {
+        const bool any_grow = __any_sync(0xffffffffu, grow);
+        float alpha = 1.f;
+        if (any_grow) {
           const float m_new = grow ? mx : m_used;
-          const float alpha = grow ? ex2((m_used - m_new) * c) : 1.f;
+          alpha = grow ? ex2((m_used - m_new) * c) : 1.f;
           l *= alpha;
           m_used = m_new;
-          if (j > 0) {
-            // the S_full arrival of this tile also covers the previous P*V MMA, so O is stable
-#pragma unroll 1
-            for (int ch = 0; ch < D / 8; ++ch) {             // rare path: kept light on registers
-              uint32_t orr[8];
-              tmem_ld8(o_addr + ch * 8, orr);
-              tmem_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 8; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
-              tmem_st8(o_addr + ch * 8, orr);
-            }
-          }
         }
         const float2 c2 = make_float2(c, c);
         const float2 nmc2 = make_float2(-m_used * c, -m_used * c);
@@ -394,14 +440,6 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           sum4[i & 3] = add2(sum4[i & 3], pr);
           const __nv_bfloat162 hh = __floats2bfloat162_rn(pr.x, pr.y);
           pk[i] = *reinterpret_cast<const uint32_t*>(&hh);
-          if (i == kBN / 4 - 1) {
-            // first 64 keys: hand them to the second MMA now
-            tmem_st32(s_addr, pk);
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t][0]));
-          }
         }
         const float2 sum2 = add2(add2(sum4[0], sum4[1]), add2(sum4[2], sum4[3]));
         l += sum2.x + sum2.y;
@@ -411,15 +449,35 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           // and its rounding error (up to 2^-9 of an output that can reach 4) would pass straight
           // into O.  The tile's largest probability is therefore entered into the sum as rounded,
           // which makes the weight of a dominant key exact; what is left is bounded by the weight
-          // of the other keys.  Same instructions as in the loop above, hence the same bits.
-          const float p_top = ex2(fmaf(mx, c, nmc2.x));
+          // of the other keys.  Same instructions as the loop above uses for that element, hence the same bits.
+          const float x_top = fmaf(mx, c, nmc2.x);
+          float p_top = ex2(x_top);
+          if (kPolyOf8 > 0 && mxf > mxs) p_top = ex2_poly2(make_float2(x_top, x_top)).x;
           l += __bfloat162float(__float2bfloat16_rn(p_top)) - p_top;
         }
-        tmem_st32(s_addr + 32, pk + 32);
+        if (j > 0) {
+          // P_t still feeds the product of the previous block, which also still adds to O_t
+          ok = __all_sync(0xffffffffu, wait_bar(&bars->p_free[t], (j - 1) & 1, bars, p.status, 11, wlim));
+          if (!ok) break;
+          tc_fence_after();
+          if (any_grow) {
+#pragma unroll 1
+            for (int ch = 0; ch < D / 8; ++ch) {             // rare path: kept light on registers
+              uint32_t orr[8];
+              tmem_ld8(o_addr + ch * 8, orr);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 8; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+              tmem_st8(o_addr + ch * 8, orr);
+            }
+          }
+        }
+        tmem_st32(p_addr, pk);
+        tmem_st32(p_addr + 32, pk + 32);
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t][1]));
+        if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t]));
       }
       if (ok) ok = __all_sync(0xffffffffu, wait_bar(&bars->o_final[t], 0, bars, p.status, 9, wlim));
       if (ok) {
@@ -477,7 +535,7 @@ EncodeTiledFn encode_fn() {
 
 template <int D>
 size_t tc_smem_bytes() {
-  return 1024 + (2 + kKStages + kVStages) * (size_t)(D / 64) * kBN * 128 + sizeof(Bars) + 64;
+  return 1024 + (2 + kKStages + kVStages) * (size_t)(D / 64) * kBN * 128 + 2 * kCopyChunk + sizeof(Bars) + 64;
 }
 
 }  // namespace

@@ -22,13 +22,15 @@
 //      after a cluster barrier, and every CTA locates the same digit.  Ties at the threshold go
 //      to the lowest candidate indices.
 //   5. the CTAs exchange their counts of kept entries, which gives every CTA its offset in the
-//      head's ascending index list; the list is written to global memory.
-//   6. stored survivors move to the front of the head's rows in rounds: in a round the cluster
-//      stages a run of list entries in shared memory, meets, then stores; the destinations of a
-//      round lie at or before its own sources and before every later round's sources.
-//   7. heads whose new rows compete (contextual heads, Eq. 10) gather their surviving new rows
-//      out of the caller's K/V; heads that keep the whole new scale leave those rows to the
-//      attention launch, which reads them from the caller's tensors and appends them itself.
+//      head's ascending index list; every entry goes straight into the shared memory of the CTA
+//      that will move it (the list never touches global memory).
+//   6. compaction in rounds: entry o of the list becomes row o of the head.  In a round every CTA
+//      stages a run of consecutive entries in shared memory (a stored survivor comes from the
+//      head's own rows, at or behind its destination; a surviving new row from the caller's K/V),
+//      the cluster meets, and the run goes out with bulk stores.  The destinations of a round lie at
+//      or before its own cache sources and before those of every later round: in place.
+//   7. heads that keep the whole new scale stop behind their stored survivors; the attention
+//      launch reads their new rows from the caller's tensors and appends them itself.
 //
 // In score-only mode the kernel stops after step 3 and writes the fp32 scores (hack_score).
 // Every mbarrier wait is bounded; a CTA whose wait gives up raises the status word, and the
@@ -116,6 +118,12 @@ __device__ __forceinline__ float ld_peer_f32(uint32_t addr) {
   float v;
   asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
   return v;
+}
+__device__ __forceinline__ void st_peer_i32(uint32_t addr, int v) {
+  asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -242,8 +250,8 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
   float* over = reinterpret_cast<float*>(sm + RING_BYTES + SUB * Q_SUB_BYTES);            // [n_over][32][128]
   uint32_t* keys = reinterpret_cast<uint32_t*>(over + (size_t)p.n_over * kMaxObs * kCkChunk);   // [cpc_max * 128]
   int32_t* pos_stage = reinterpret_cast<int32_t*>(keys + (size_t)p.cpc_max * kCkChunk);        // [stage_rows]
-  int32_t* src_stage = pos_stage + p.stage_rows;                                                // [stage_rows]
-  CkShared* sh = reinterpret_cast<CkShared*>(src_stage + p.stage_rows);
+  int32_t* src_all = pos_stage + p.stage_rows;              // [cpc_max * 128 + stage_rows]: this CTA's list entries of every round
+  CkShared* sh = reinterpret_cast<CkShared*>(src_all + (size_t)p.cpc_max * kCkChunk + p.stage_rows);
   float* fold_m = reinterpret_cast<float*>(sm);           // [32][128], reuses the ring
   float* fold_l = fold_m + kMaxObs * kCkChunk;
 
@@ -445,12 +453,14 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
   const bool aborted = sh->sh_abort != 0;                   // the same value in every CTA of the cluster
 
   // ------------------------------------------------------------------ 3. scores, pass 2
-  if (!aborted && warp >= 2 && warp < 6) {
+  if (!aborted) {
+    // all eight warps: warps 2-5 take the even chunks, warps 6, 7, 0, 1 (the same four lane quadrants)
+    // the odd ones; a key's 32 terms are added in the same order by either set
     float rm[kMaxObs], rl[kMaxObs];
 #pragma unroll
     for (int i = 0; i < kMaxObs; ++i) { rm[i] = sh->row_m[i]; rl[i] = sh->row_inv_l[i]; }
     const bool structural = ctx == 0;
-    for (int i = 0; i < n_run; ++i) {
+    for (int i = (warp >= 2 && warp < 6) ? 0 : 1; i < n_run; i += 2) {
       // a chunk of protected candidates only (the new scale of a structural head) is kept whatever
       // its scores are; they are formed only when the caller wants them
       if (!p.scores && structural && a.protect_new && c_begin + i >= n_sc) {
@@ -576,78 +586,97 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
         }
     }
     const int n_old = gt_old_all + min(eq_old_all, need);     // survivors that were already stored
-    // heads that keep the whole new scale need only the stored survivors' part of the list
+    // Entry o of the head's ascending list is candidate j.  Entry o becomes row o of the head, and
+    // rows are compacted in rounds of CL * S consecutive entries, CTA `rk` of the cluster staging S
+    // of them: the entry goes straight into that CTA's shared memory.  Heads that keep the whole new
+    // scale need only their stored survivors (the attention launch appends the rest).
     const bool attend_appends = a.seg_new[ctx] != 0;
-    int32_t* list = p.idx + (size_t)bh * a.kept_stride;
+    const int n_rows = attend_appends ? n_old : n_keep;
+    const int S = p.stage_rows, RS = CL * S;
+    auto deliver = [&](int o, int j) {
+      if (o < n_rows && dbg_ok(o >= 0 && o < n_keep, a.status, 9)) {
+        const int t = o / RS, w = o - t * RS, rk = w / S, lr = w - rk * S;
+        st_peer_i32(peer_addr(&src_all[t * S + lr], rk), j);
+      }
+    };
     for (int e = 0; e < per; ++e) {
       const int slot = tid * per + e;
       int j;
       if (slot < n_slots && slot_info(slot, j)) {
         const uint32_t k = keys[slot];
         if (k > thr) {
-          const int o = gt_before + min(eq_before, need);
-          if (!(attend_appends && j >= stored) && dbg_ok(o >= 0 && o < n_keep, a.status, 9)) list[o] = j;
+          deliver(gt_before + min(eq_before, need), j);
           ++gt_before;
         } else if (k == thr) {
-          if (eq_before < need && !(attend_appends && j >= stored) && dbg_ok(gt_before + eq_before < n_keep, a.status, 9))
-            list[gt_before + eq_before] = j;
+          if (eq_before < need) deliver(gt_before + eq_before, j);
           ++eq_before;
         }
       }
     }
-    __threadfence();
     __syncthreads();
-    cluster_sync();                                           // the list is complete and visible in the cluster
+    cluster_sync();                                           // every CTA holds its part of the list
 
     // ---------------------------------------------------------------- 6. and 7. compaction in rounds
-    // Entry r of the list becomes row r of the head: a stored survivor moves forward (its source
-    // is a row of the head at or behind r), a surviving new row comes out of the caller's K/V.
-    // In a round the cluster stages a run of consecutive entries in shared memory, meets, and then
-    // stores: the destinations of a round lie at or before its own cache sources and before the
-    // cache sources of every later round, so nothing is overwritten before it has been read.
-    // Heads that keep the whole new scale stop behind their stored survivors.
+    // A stored survivor moves forward (its source is a row of the head at or behind its
+    // destination), a surviving new row comes out of the caller's K/V.  In a round every CTA stages
+    // its S entries in shared memory, the cluster meets, and the rows go out with bulk stores (the
+    // destinations of a CTA are one contiguous run).  The destinations of a round lie at or before
+    // its own cache sources and before the cache sources of every later round, so nothing is
+    // overwritten before it has been read: in place, no second buffer.
     const size_t off = a.row_off[bh];
     uint4* kp = reinterpret_cast<uint4*>(a.k_plane) + off * PIECES;
     uint4* vp = reinterpret_cast<uint4*>(a.v_plane) + off * PIECES;
     int32_t* pos = a.pos_plane + off;
     const uint4* kn = p.k_new + (size_t)bh * n_new * PIECES;
     const uint4* vn = p.v_new + (size_t)bh * n_new * PIECES;
-    const int n_rows = attend_appends ? n_old : n_keep;
-    const int S = p.stage_rows;
-    for (int r0 = 0; r0 < n_rows; r0 += CL * S) {
+    constexpr uint32_t ROWB = PIECES * 16;
+    const uint32_t v_base = base + (uint32_t)S * ROWB;       // staging: S key rows, then S value rows
+    int t = 0;
+    for (int r0 = 0; r0 < n_rows; r0 += RS, ++t) {
       const int first = r0 + rank * S;
       const int rows = max(0, min(S, n_rows - first));
-      for (int lr = tid; lr < rows; lr += kCkThreads) {
-        int src = list[first + lr];
-        // a checked build turns an entry outside [dst, candidates) into "stays where it is"
-        if (!dbg_ok(src >= first + lr && src < stored + n_new && first + lr < a.cap[ctx], a.status, 10)) src = first + lr;
-        src_stage[lr] = src;
-        pos_stage[lr] = src < stored ? pos[src] : a.pos_base + (src - stored);
-      }
-      __syncthreads();
-      for (int v = tid; v < rows * PIECES; v += kCkThreads) {
-        const int lr = v / PIECES, piece = v % PIECES;
-        const int src = src_stage[lr];
-        if (src >= stored || src != first + lr) {            // a stored row that stays where it is needs nothing
+      const int32_t* srcs = src_all + t * S;
+      // ascending entries with source >= destination: if the last stored row of the slice stays
+      // where it is, so does every row of the slice
+      const bool moving = rows > 0 && !(srcs[rows - 1] == first + rows - 1 && srcs[rows - 1] < stored);
+      if (moving) {
+        for (int v = tid; v < rows * PIECES; v += kCkThreads) {
+          const int lr = v / PIECES, piece = v % PIECES;
+          int src = srcs[lr];
+          // a checked build turns an entry outside [destination, candidates) into "stays where it is"
+          if (!dbg_ok(src >= first + lr && src < stored + n_new && first + lr < a.cap[ctx], a.status, 10)) src = first + lr < stored ? first + lr : stored;
           const uint4* ks = src < stored ? kp + (size_t)src * PIECES : kn + (size_t)(src - stored) * PIECES;
           const uint4* vs = src < stored ? vp + (size_t)src * PIECES : vn + (size_t)(src - stored) * PIECES;
-          cp_async16(base + (uint32_t)((lr * 2) * PIECES + piece) * 16, ks + piece);
-          cp_async16(base + (uint32_t)((lr * 2 + 1) * PIECES + piece) * 16, vs + piece);
+          cp_async16(base + (uint32_t)lr * ROWB + piece * 16, ks + piece);
+          cp_async16(v_base + (uint32_t)lr * ROWB + piece * 16, vs + piece);
         }
+        for (int lr = tid; lr < rows; lr += kCkThreads) {
+          const int src = srcs[lr];
+          if (src < stored) cp_async4(smem_u32(&pos_stage[lr]), pos + max(src, 0));
+          else pos_stage[lr] = a.pos_base + (src - stored);
+        }
+        cp_async_wait_all();
+        fence_proxy_async();                                  // the bulk stores below read what these threads wrote
       }
-      cp_async_wait_all();
       __syncthreads();
       cluster_sync();                                         // every source of this round has been read
-      for (int v = tid; v < rows * PIECES; v += kCkThreads) {
-        const int lr = v / PIECES, piece = v % PIECES;
-        if (src_stage[lr] >= stored || src_stage[lr] != first + lr) {
-          kp[(size_t)(first + lr) * PIECES + piece] = *reinterpret_cast<const uint4*>(sm + (size_t)((lr * 2) * PIECES + piece) * 16);
-          vp[(size_t)(first + lr) * PIECES + piece] = *reinterpret_cast<const uint4*>(sm + (size_t)((lr * 2 + 1) * PIECES + piece) * 16);
+      if (moving) {
+        if (tid == 0) {
+          constexpr uint32_t kPiece = 32768;                  // bytes per bulk store
+          const uint32_t bytes = (uint32_t)rows * ROWB;
+          for (uint32_t o = 0; o < bytes; o += kPiece) {
+            const uint32_t n = min(kPiece, bytes - o);
+            bulk_store(reinterpret_cast<unsigned char*>(kp + (size_t)first * PIECES) + o, base + o, n);
+            bulk_store(reinterpret_cast<unsigned char*>(vp + (size_t)first * PIECES) + o, v_base + o, n);
+          }
+          bulk_commit();
         }
+        for (int lr = tid; lr < rows; lr += kCkThreads) pos[first + lr] = pos_stage[lr];
+        if (tid == 0) bulk_wait_read<0>();                    // the staging area is reused by the next round
       }
-      for (int lr = tid; lr < rows; lr += kCkThreads) pos[first + lr] = pos_stage[lr];
-      __syncthreads();                                        // the staging area is reused by the next round
+      __syncthreads();
     }
+    if (tid == 0) bulk_wait<0>();                             // the rows are in place before the CTA leaves
   }
   // no CTA leaves while another may still read its shared memory
   cluster_sync();
@@ -663,7 +692,7 @@ template <int D>
 size_t ck_smem_bytes(const CkParams& p) {
   return 1024 + (size_t)p.stages * (D / 64) * kCkChunk * 128 + (size_t)(D / 64) * kMaxObs * 128 +
          (size_t)p.n_over * kMaxObs * kCkChunk * sizeof(float) + (size_t)p.cpc_max * kCkChunk * sizeof(uint32_t) +
-         2 * (size_t)p.stage_rows * sizeof(int32_t) + sizeof(CkShared) + 64;
+         (2 * (size_t)p.stage_rows + (size_t)p.cpc_max * kCkChunk) * sizeof(int32_t) + sizeof(CkShared) + 64;
 }
 
 // Ring depth and staging rows for this launch: as many key tiles in flight as the CTA has chunks

@@ -8,29 +8,13 @@
 #include <algorithm>
 
 #include "hack_internal.h"
+#include "score_simt.cuh"
 
 namespace hack {
 namespace {
 
-template <typename T> struct Elem;
-template <> struct Elem<float> {
-  static constexpr int kPerVec = 4;  // elements per 16 bytes
-  __device__ static void unpack(const uint4& v, float* f) {
-    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
-    f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
-  }
-};
-template <> struct Elem<__nv_bfloat16> {
-  static constexpr int kPerVec = 8;
-  __device__ static void unpack(const uint4& v, float* f) {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      f[2 * i] = __uint_as_float(w[i] << 16);
-      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-  }
-};
+using simt::Elem;
+static_assert(simt::kObs == kMaxObs && simt::kChunk == kScoreChunk, "the shared SIMT body is built for these sizes");
 
 // Row pointer of candidate j of head bh: stored entries first, then the new scale's tokens.
 template <typename T>
@@ -45,98 +29,21 @@ __global__ void __launch_bounds__(kScoreChunk)
 score_logits_kernel(const StepArgs a, const T* __restrict__ q, const T* __restrict__ k_new,
                     float* __restrict__ logits, float* __restrict__ partials, int max_chunks) {
   pdl_wait();
-  constexpr int VEC = Elem<T>::kPerVec;
-  constexpr int ROWV = D / VEC;                 // 16-byte vectors per row
-  constexpr int KROW = ROWV + 1;                // padded row stride (in vectors) of the key tile
   const int bh = blockIdx.y;
   const int ctx = a.is_ctx[bh % a.n_heads];
   if (!a.trig[ctx]) return;
   const int cand = a.cand[ctx], stored = a.stored[ctx];
   const int j0 = blockIdx.x * kScoreChunk;
   if (j0 >= cand) return;
-  const int tid = threadIdx.x;
-
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* qs = reinterpret_cast<float*>(smem_raw);                       // [32][D]
-  uint4* ks = reinterpret_cast<uint4*>(smem_raw + kMaxObs * D * 4);     // [128][KROW]
-  float* zt = reinterpret_cast<float*>(ks);                             // reused: [32][128]
-
   const T* kp = static_cast<const T*>(a.k_plane);
-  // observation rows: floor(m * N_k / n) under the uniform rule
-  for (int v = tid; v < kMaxObs * ROWV; v += kScoreChunk) {
-    const int i = v / ROWV, c = v % ROWV;
-    float f[VEC];
-    if (i < a.n_obs_rows) {
-      const int row = obs_row(a, i);
-      const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)bh * a.n_new + row) * D + c * VEC);
-      Elem<T>::unpack(raw, f);
-    } else {
-#pragma unroll
-      for (int e = 0; e < VEC; ++e) f[e] = 0.f;
-    }
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) qs[i * D + c * VEC + e] = f[e];
-  }
-  for (int v = tid; v < kScoreChunk * ROWV; v += kScoreChunk) {
-    const int r = v / ROWV, c = v % ROWV;
-    const int j = j0 + r;
-    uint4 raw = make_uint4(0, 0, 0, 0);
-    if (j < cand) raw = *reinterpret_cast<const uint4*>(cand_row(a, kp, k_new, bh, stored, j) + c * VEC);
-    ks[r * KROW + c] = raw;
-  }
-  __syncthreads();
-
-  float acc[kMaxObs];
-#pragma unroll
-  for (int i = 0; i < kMaxObs; ++i) acc[i] = 0.f;
-  for (int c = 0; c < ROWV; ++c) {
-    float kf[VEC];
-    Elem<T>::unpack(ks[tid * KROW + c], kf);
-#pragma unroll
-    for (int i = 0; i < kMaxObs; ++i) {
-      const float4* qv = reinterpret_cast<const float4*>(qs + i * D + c * VEC);
-#pragma unroll
-      for (int e4 = 0; e4 < VEC / 4; ++e4) {
-        const float4 qq = qv[e4];
-        acc[i] = fmaf(qq.x, kf[4 * e4 + 0], acc[i]);
-        acc[i] = fmaf(qq.y, kf[4 * e4 + 1], acc[i]);
-        acc[i] = fmaf(qq.z, kf[4 * e4 + 2], acc[i]);
-        acc[i] = fmaf(qq.w, kf[4 * e4 + 3], acc[i]);
-      }
-    }
-  }
-  __syncthreads();                     // everyone is done with the key tile; reuse it for logits
-  const bool valid = (j0 + tid) < cand;
-#pragma unroll
-  for (int i = 0; i < kMaxObs; ++i) zt[i * kScoreChunk + tid] = valid ? acc[i] * a.sm_scale : -INFINITY;
-  __syncthreads();
-
-  // each warp owns 8 observation rows: store logits (coalesced) and reduce (max, sum-exp)
-  const int warp = tid >> 5, lane = tid & 31;
   const int chunk = blockIdx.x;
-  for (int i = warp; i < a.n_obs_rows; i += kScoreChunk / 32) {
-    float z[4];
-    float m = -INFINITY;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      z[u] = zt[i * kScoreChunk + u * 32 + lane];
-      m = fmaxf(m, z[u]);
-      const int j = j0 + u * 32 + lane;
-      if (j < cand) logits[((size_t)bh * kMaxObs + i) * a.cand_stride + j] = z[u];
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    float l = 0.f;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) l += expf(z[u] - m);      // exp(-inf) = 0 for padding
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-    if (lane == 0) {
-      float* p = partials + (((size_t)bh * max_chunks + chunk) * kMaxObs + i) * 2;
-      p[0] = m;
-      p[1] = l;
-    }
-  }
+  simt::chunk_logits<T, D>(
+      smem_raw, j0, cand, a.n_obs_rows, a.sm_scale,
+      [&](int i) { return q + ((size_t)bh * a.n_new + obs_row(a, i)) * D; },     // floor(m * N_k / n) under the uniform rule
+      [&](int j) { return cand_row(a, kp, k_new, bh, stored, j); },
+      [&](int i, int j) -> float& { return logits[((size_t)bh * kMaxObs + i) * a.cand_stride + j]; },
+      [&](int i) { return partials + (((size_t)bh * max_chunks + chunk) * kMaxObs + i) * 2; });
 }
 
 __global__ void __launch_bounds__(256)
@@ -151,26 +58,13 @@ score_reduce_kernel(const StepArgs a, const float* __restrict__ logits,
   if (j0 >= cand) return;
   __shared__ float row_m[kMaxObs], row_inv_l[kMaxObs];
   const int n_chunks = (cand + kScoreChunk - 1) / kScoreChunk;
-  if (threadIdx.x < a.n_obs_rows) {
-    const int i = threadIdx.x;
-    const float* p = partials + ((size_t)bh * max_chunks * kMaxObs + i) * 2;
-    float m = -INFINITY;
-    for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, p[(size_t)c * kMaxObs * 2]);
-    float l = 0.f;
-    for (int c = 0; c < n_chunks; ++c)
-      l += p[(size_t)c * kMaxObs * 2 + 1] * expf(p[(size_t)c * kMaxObs * 2] - m);
-    row_m[i] = m;
-    row_inv_l[i] = 1.f / l;
-  }
-  __syncthreads();
-  const int j = j0 + threadIdx.x;
-  if (j >= cand) return;
-  float s = 0.f;
-  for (int i = 0; i < a.n_obs_rows; ++i) {
-    const float z = logits[((size_t)bh * kMaxObs + i) * a.cand_stride + j];
-    s += expf(z - row_m[i]) * row_inv_l[i];
-  }
-  float* dst = scores + (size_t)bh * a.cand_stride + j;
+  float s;
+  if (!simt::column_scores(
+          row_m, row_inv_l, j0, cand, a.n_obs_rows, n_chunks,
+          [&](int c, int i) { return partials + (((size_t)bh * max_chunks + c) * kMaxObs + i) * 2; },
+          [&](int i, int j) { return logits[((size_t)bh * kMaxObs + i) * a.cand_stride + j]; }, s))
+    return;
+  float* dst = scores + (size_t)bh * a.cand_stride + j0 + threadIdx.x;
   *dst = a.score_accumulate ? *dst + s : s;
 }
 
@@ -179,9 +73,7 @@ int launch_score_t(const StepArgs& a, const void* q, const void* k_new, float* s
                    const Scratch& s, cudaStream_t st) {
   const int max_cand = a.cand[0] * a.trig[0] > a.cand[1] * a.trig[1] ? a.cand[0] : a.cand[1];
   const int bh = a.batch * a.n_heads;
-  constexpr int VEC = Elem<T>::kPerVec;
-  const size_t smem = (size_t)kMaxObs * D * 4 +
-                      (size_t)kScoreChunk * (D / VEC + 1) * 16;   // >= 32*128*4 for the logit tile
+  const size_t smem = simt::logits_smem_bytes<T, D>();
   if (!allow_dynamic_smem(score_logits_kernel<T, D>, smem)) return -1;
   dim3 g1((max_cand + kScoreChunk - 1) / kScoreChunk, bh);
   launch_k(score_logits_kernel<T, D>, g1, kScoreChunk, smem, st, 

@@ -19,11 +19,13 @@
 #include <mutex>
 
 #include "hack_internal.h"
+#include "score_simt.cuh"
 
 namespace hack {
 namespace {
 
-constexpr int kChunk = 128;                               // candidate keys per CTA in pass 1
+constexpr int kChunk = simt::kChunk;                      // candidate keys per CTA in pass 1
+static_assert(simt::kObs == kMaxObs, "the shared SIMT body is built for 32 observation rows");
 constexpr long long kMaxLogitRows = 65536;                // limit on n_rows * n_cand
 constexpr int kMaxRows = 512;                             // limit on n_rows (batch * heads)
 constexpr long long kLogitFloats = kMaxLogitRows * kMaxObs;                     // 2 Mi floats
@@ -34,143 +36,39 @@ constexpr long long kScratchFloats = kLogitFloats + kPartialFloats;
 // cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) float g_noalloc_scratch[kScratchFloats];
 
-template <typename T> struct Ld;
-template <> struct Ld<float> {
-  static constexpr int kPerVec = 4;
-  __device__ static void unpack(const uint4& v, float* f) {
-    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
-    f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
-  }
-};
-template <> struct Ld<__nv_bfloat16> {
-  static constexpr int kPerVec = 8;
-  __device__ static void unpack(const uint4& v, float* f) {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      f[2 * i] = __uint_as_float(w[i] << 16);
-      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-  }
-};
-
 struct DenseArgs {
   int n_queries, n_cand, n_obs_rows, chunks_per_row;
   float sm_scale;
 };
 
-// Pass 1: logits of 128 candidates of one row-block against the observation rows, plus the
-// (max, sum-exp) of every observation row over this chunk.
+// Pass 1 and pass 2 of the shared SIMT body (score_simt.cuh) on dense tensors: row-block `row` has
+// n_queries query rows (observation row i = floor(i * n_queries / n)) and n_cand candidate keys.
 template <typename T, int D>
 __global__ void __launch_bounds__(kChunk)
 noalloc_logits_kernel(const DenseArgs a, const T* __restrict__ q, const T* __restrict__ k_cand,
                       float* __restrict__ logits, float* __restrict__ partials) {
-  constexpr int VEC = Ld<T>::kPerVec;
-  constexpr int ROWV = D / VEC;
-  constexpr int KROW = ROWV + 1;
   const int row = blockIdx.y;
-  const int j0 = blockIdx.x * kChunk;
-  const int tid = threadIdx.x;
+  const int chunk = blockIdx.x;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* qs = reinterpret_cast<float*>(smem_raw);
-  uint4* ks = reinterpret_cast<uint4*>(smem_raw + kMaxObs * D * 4);
-  float* zt = reinterpret_cast<float*>(ks);
-
-  for (int v = tid; v < kMaxObs * ROWV; v += kChunk) {
-    const int i = v / ROWV, c = v % ROWV;
-    float f[VEC];
-    if (i < a.n_obs_rows) {
-      const int qrow = (int)(((long long)i * a.n_queries) / a.n_obs_rows);
-      Ld<T>::unpack(*reinterpret_cast<const uint4*>(q + ((size_t)row * a.n_queries + qrow) * D + c * VEC), f);
-    } else {
-#pragma unroll
-      for (int e = 0; e < VEC; ++e) f[e] = 0.f;
-    }
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) qs[i * D + c * VEC + e] = f[e];
-  }
-  for (int v = tid; v < kChunk * ROWV; v += kChunk) {
-    const int r = v / ROWV, c = v % ROWV;
-    const int j = j0 + r;
-    uint4 raw = make_uint4(0, 0, 0, 0);
-    if (j < a.n_cand) raw = *reinterpret_cast<const uint4*>(k_cand + ((size_t)row * a.n_cand + j) * D + c * VEC);
-    ks[r * KROW + c] = raw;
-  }
-  __syncthreads();
-  float acc[kMaxObs];
-#pragma unroll
-  for (int i = 0; i < kMaxObs; ++i) acc[i] = 0.f;
-  for (int c = 0; c < ROWV; ++c) {
-    float kf[VEC];
-    Ld<T>::unpack(ks[tid * KROW + c], kf);
-#pragma unroll
-    for (int i = 0; i < kMaxObs; ++i) {
-      const float4* qv = reinterpret_cast<const float4*>(qs + i * D + c * VEC);
-#pragma unroll
-      for (int e4 = 0; e4 < VEC / 4; ++e4) {
-        const float4 qq = qv[e4];
-        acc[i] = fmaf(qq.x, kf[4 * e4 + 0], acc[i]);
-        acc[i] = fmaf(qq.y, kf[4 * e4 + 1], acc[i]);
-        acc[i] = fmaf(qq.z, kf[4 * e4 + 2], acc[i]);
-        acc[i] = fmaf(qq.w, kf[4 * e4 + 3], acc[i]);
-      }
-    }
-  }
-  __syncthreads();
-  const bool valid = (j0 + tid) < a.n_cand;
-#pragma unroll
-  for (int i = 0; i < kMaxObs; ++i) zt[i * kChunk + tid] = valid ? acc[i] * a.sm_scale : -INFINITY;
-  __syncthreads();
-  const int warp = tid >> 5, lane = tid & 31;
-  for (int i = warp; i < a.n_obs_rows; i += kChunk / 32) {
-    float z[4];
-    float m = -INFINITY;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      z[u] = zt[i * kChunk + u * 32 + lane];
-      m = fmaxf(m, z[u]);
-      const int j = j0 + u * 32 + lane;
-      if (j < a.n_cand) logits[((size_t)row * kMaxObs + i) * a.n_cand + j] = z[u];
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    float l = 0.f;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) l += expf(z[u] - m);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-    if (lane == 0) {
-      float* p = partials + (((size_t)row * a.chunks_per_row + blockIdx.x) * kMaxObs + i) * 2;
-      p[0] = m;
-      p[1] = l;
-    }
-  }
+  simt::chunk_logits<T, D>(
+      smem_raw, chunk * kChunk, a.n_cand, a.n_obs_rows, a.sm_scale,
+      [&](int i) { return q + ((size_t)row * a.n_queries + (int)(((long long)i * a.n_queries) / a.n_obs_rows)) * D; },
+      [&](int j) { return k_cand + ((size_t)row * a.n_cand + j) * D; },
+      [&](int i, int j) -> float& { return logits[((size_t)row * kMaxObs + i) * a.n_cand + j]; },
+      [&](int i) { return partials + (((size_t)row * a.chunks_per_row + chunk) * kMaxObs + i) * 2; });
 }
 
-// Pass 2: merge the chunk statistics into full-softmax row statistics and reduce each column.
 __global__ void __launch_bounds__(256)
 noalloc_reduce_kernel(const DenseArgs a, const float* __restrict__ logits,
                       const float* __restrict__ partials, float* __restrict__ scores, int score_stride) {
   const int row = blockIdx.y;
   __shared__ float row_m[kMaxObs], row_inv_l[kMaxObs];
-  if (threadIdx.x < a.n_obs_rows) {
-    const int i = threadIdx.x;
-    const float* p = partials + ((size_t)row * a.chunks_per_row * kMaxObs + i) * 2;
-    float m = -INFINITY;
-    for (int c = 0; c < a.chunks_per_row; ++c) m = fmaxf(m, p[(size_t)c * kMaxObs * 2]);
-    float l = 0.f;
-    for (int c = 0; c < a.chunks_per_row; ++c)
-      l += p[(size_t)c * kMaxObs * 2 + 1] * expf(p[(size_t)c * kMaxObs * 2] - m);
-    row_m[i] = m;
-    row_inv_l[i] = 1.f / l;
-  }
-  __syncthreads();
-  const int j = blockIdx.x * 256 + threadIdx.x;
-  if (j >= a.n_cand) return;
-  float s = 0.f;
-  for (int i = 0; i < a.n_obs_rows; ++i)
-    s += expf(logits[((size_t)row * kMaxObs + i) * a.n_cand + j] - row_m[i]) * row_inv_l[i];
-  scores[(size_t)row * score_stride + j] = s;
+  float s;
+  if (simt::column_scores(
+          row_m, row_inv_l, blockIdx.x * 256, a.n_cand, a.n_obs_rows, a.chunks_per_row,
+          [&](int c, int i) { return partials + (((size_t)row * a.chunks_per_row + c) * kMaxObs + i) * 2; },
+          [&](int i, int j) { return logits[((size_t)row * kMaxObs + i) * a.n_cand + j]; }, s))
+    scores[(size_t)row * score_stride + blockIdx.x * 256 + threadIdx.x] = s;
 }
 
 // One scratch address per device, resolved on the first call made with that device current.
@@ -180,8 +78,7 @@ float* g_scratch_ptr[64] = {nullptr};
 template <typename T, int D>
 cudaError_t run(const DenseArgs& a, int n_rows, const void* q, const void* k, float* scratch,
                 float* scores, int score_stride, cudaStream_t st) {
-  constexpr int VEC = Ld<T>::kPerVec;
-  const size_t smem = (size_t)kMaxObs * D * 4 + (size_t)kChunk * (D / VEC + 1) * 16;
+  const size_t smem = simt::logits_smem_bytes<T, D>();
   // opt-in to more than 48 KB of dynamic shared memory, once per (kernel, device)
   if (!allow_dynamic_smem(noalloc_logits_kernel<T, D>, smem)) return cudaErrorInvalidValue;
   float* logits = scratch;

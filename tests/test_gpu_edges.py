@@ -171,3 +171,61 @@ def test_graph_replay_reproduces_direct_calls():
         assert direct.hack_get_lengths(l) == replayed.hack_get_lengths(l)
     direct.close()
     replayed.close()
+
+
+def test_kept_list_beyond_65536_entries():
+    """A budget above 65 536 entries: the compaction has to find the boundary between stored
+    survivors and new rows in a kept list longer than its probe round covers at once.  Schedule
+    (1, 2, 258, 30): the third scale brings 66 564 tokens and is only appended; the fourth exceeds
+    the budget of 66 600, so 66 600 of 67 469 candidates survive.  Scores, index list, stored rows
+    and positions are compared at that step, and its attention output (900 queries) as well; the
+    oracle skips the output of the huge third scale (a 66 564 x 66 569 matrix in fp64)."""
+    import numpy as np
+    import torch
+    import paper_2504_09261_b200 as hb
+    from oracle import hack_oracle as ho
+    from workloads import SyntheticQKV
+    from tests.parity_util import OUT_TOL, SCORE_ATOL, SCORE_RTOL, _rows_bytes
+    cfg = _custom(1, n_heads=2, batch=1, sides=(1, 2, 258, 30))
+    budget = 66600
+    dev = torch.device("cuda:0")
+    gen = SyntheticQKV(cfg, device=dev)
+    mask = gen.head_is_contextual.numpy()
+    cache = hb.HackCache(1, cfg.n_heads, cfg.head_dim, 1, cfg.sides, hb.HACK_BF16, mask, budget, budget,
+                         overflow_policy=hb.HACK_OVERFLOW_COMPETE)
+    orc = ho.HackOracle(1, cfg.n_heads, 1, cfg.head_dim, cfg.sides, mask, budget, budget,
+                        overflow_policy=ho.COMPETE)
+    bh = cfg.n_heads
+    scores = torch.zeros((bh, cache.cand_stride), dtype=torch.float32, device=dev)
+    idx = torch.full((bh, cache.kept_stride), -1, dtype=torch.int32, device=dev)
+    for k in range(cfg.n_scales):
+        q, kk, v = gen.qkv(0, k)
+        out = torch.full_like(q, float("nan"))
+        info = cache.hack_step_info(0, k)
+        last = k == cfg.n_scales - 1
+        assert bool(info.triggered_c and info.triggered_s) == last
+        cache.hack_score(0, k, q, kk, scores)
+        cache.hack_select(0, k, scores, idx)
+        cache.hack_compact(0, k, idx, kk, v)
+        cache.hack_attend(0, k, q, out)
+        torch.cuda.synchronize()
+        cache.hack_poll_status()
+        q64, k64, v64 = (t.to(torch.float64).cpu().numpy() for t in (q, kk, v))
+        override = {(0, h): scores[h, :info.cand_c].cpu().numpy().astype(np.float64) for h in range(bh)} if last else None
+        o_ref, recs = orc.scale_step(0, k, q64, k64, v64, scores_override=override, need_output=last)
+        if not last:
+            continue
+        assert info.kept_c == budget and info.kept_s == budget and info.cand_c == 67469
+        for h in range(bh):
+            rec = recs[(0, h)]
+            sg = scores[h, :info.cand_c].cpu().numpy().astype(np.float64)
+            den = SCORE_RTOL * np.maximum(np.abs(sg), np.abs(rec.scores)) + SCORE_ATOL
+            assert np.all(np.abs(sg - rec.scores) <= den)
+            assert np.array_equal(idx[h, :budget].cpu().numpy().astype(np.int64), rec.keep)
+            st = orc.state[0][0][h]
+            assert np.array_equal(np.frombuffer(cache.hack_read_head(0, 0, h, 2), dtype=np.int32).astype(np.int64), st.pos)
+            assert cache.hack_read_head(0, 0, h, 0) == _rows_bytes(st.k, torch.bfloat16)
+            assert cache.hack_read_head(0, 0, h, 1) == _rows_bytes(st.v, torch.bfloat16)
+            d = float(np.max(np.abs(out[0, h].to(torch.float64).cpu().numpy() - o_ref[0, h])))
+            assert d <= OUT_TOL["bf16"], f"head {h}: attention output off by {d:.3e}"
+    cache.close()

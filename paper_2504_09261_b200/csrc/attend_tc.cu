@@ -555,7 +555,7 @@ bool make_rows_map(void* out_map, const void* base, uint64_t rows, int head_dim)
 
 int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
                      const void* q, void* out, float* row_stats, const void* k_new, const void* v_new,
-                     int n_heads_served, cudaStream_t st) {
+                     int n_heads_served, bool shares_gpu, cudaStream_t st) {
   CUtensorMap tm_q;
   if (!make_rows_map(&tm_q, q, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) {
     set_error("attention: cuTensorMapEncodeTiled failed for the queries");
@@ -568,8 +568,8 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
   // n_heads_served < all heads: only the first heads of head_order (those of one type) are served
   const int heads = n_heads_served > 0 ? n_heads_served : a.batch * a.n_heads;
   // one query tile per CTA while that still fits one wave: twice the CTAs, no idle SMs; a launch
-  // that serves one head type shares the GPU with the other type's kernels and keeps two
-  p.tiles_per_cta = (n_heads_served == 0 && n_tiles * heads <= sm_count()) ? 1 : 2;
+  // that shares the GPU with the other head type's compression keeps two
+  p.tiles_per_cta = (!shares_gpu && n_tiles * heads <= sm_count()) ? 1 : 2;
   p.n_pairs = (n_tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
   const CUtensorMap& tk = *static_cast<const CUtensorMap*>(k_map);
   const CUtensorMap& tv = *static_cast<const CUtensorMap*>(v_map);

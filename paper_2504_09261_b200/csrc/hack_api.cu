@@ -54,7 +54,7 @@ bool attend_tc_serves(const StepArgs& a, int dtype) {
 
 int launch_attend(const StepArgs& a, int dtype, const void* q, void* out, cudaStream_t st) {
   if (attend_tc_serves(a, dtype))
-    return launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, nullptr, nullptr, 0, st);
+    return launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, nullptr, nullptr, 0, false, st);
   return launch_attend_simt(a, dtype, q, out, st);
 }
 
@@ -692,7 +692,8 @@ hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const 
 // from the caller's tensors and appended by the attention kernel itself.
 static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void* q, void* out, float* sigma,
                                  cudaStream_t st, const void* k_new = nullptr, const void* v_new = nullptr,
-                                 const int* seg_new = nullptr, int only_type = -1, bool finish = true) {
+                                 const int* seg_new = nullptr, int only_type = -1, bool finish = true,
+                                 bool shares_gpu = false) {
   // lengths are already those after compaction
   LayerState& ls = c->layers[layer];
   hack_step_info_t p{};
@@ -708,7 +709,7 @@ static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void
     // Eq. 6 needs the statistics of every softmax row; the tensor-core attention kernel leaves them
     if (!hack::attend_tc_serves(a, c->cfg.dtype))
       return fail(HACK_ERR_UNSUPPORTED, "hack_attend_variance needs a bf16 cache and a scale of at least 32 tokens (128 query rows over all heads)");
-    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, c->attn_row_stats, nullptr, nullptr, 0, st);
+    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, c->attn_row_stats, nullptr, nullptr, 0, false, st);
     if (n >= 0) {
       const int m = hack::launch_attention_variance(a, q, c->attn_row_stats, c->attn_block_var, c->var_blocks, sigma, st);
       n = m < 0 ? m : n + m;
@@ -722,7 +723,7 @@ static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void
       served = only_type == 1 ? n_ctx : bh - n_ctx;
       a.head_order = c->head_order + ((size_t)layer * 2 + only_type) * bh;
     }
-    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, k_new, v_new, served, st);
+    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, k_new, v_new, served, shares_gpu, st);
   } else {
     n = hack::launch_attend(a, c->cfg.dtype, q, out, st);
   }
@@ -839,7 +840,7 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
     if (compressed) {
       c->launches += n;
       advance_after_compact(c, layer, p);
-      s = attend_impl(c, layer, scale, q, out, nullptr, c->side_stream, k, v, seg_new, 1 - trig_type, false);
+      s = attend_impl(c, layer, scale, q, out, nullptr, c->side_stream, k, v, seg_new, 1 - trig_type, false, true);
       if (s == HACK_OK) s = attend_impl(c, layer, scale, q, out, nullptr, st, k, v, seg_new, trig_type, true);
     }
     // the side stream always comes back to the caller's stream (it may be part of a capture)

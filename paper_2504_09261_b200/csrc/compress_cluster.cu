@@ -17,18 +17,20 @@
 //   3. scores, pass 2: the logits are read back from tensor / shared memory (no second key
 //      load, no second MMA) and s_j = sum_i exp(z_ij - m_i) / l_i becomes an order-preserving
 //      32-bit key in shared memory (protected candidates of structural heads carry the top key).
-//   4. exact radix select over the cluster: four passes of 8-bit digits; every CTA builds the
-//      histogram of its own keys, the histograms are added through distributed shared memory
-//      after a cluster barrier, and every CTA locates the same digit.  Ties at the threshold go
-//      to the lowest candidate indices.
+//   4. exact radix select over the cluster: digits of 12, 12 and 8 bits; every CTA builds the
+//      histogram of its own keys (the first one while it forms them), the histograms are added
+//      through distributed shared memory after a cluster barrier, and every CTA locates the same
+//      digit.  The select stops once all entries left in the located bin survive.  Ties at the
+//      threshold go to the lowest candidate indices.
 //   5. the CTAs exchange their counts of kept entries, which gives every CTA its offset in the
 //      head's ascending index list; every entry goes straight into the shared memory of the CTA
 //      that will move it (the list never touches global memory).
 //   6. compaction in rounds: entry o of the list becomes row o of the head.  In a round every CTA
-//      stages a run of consecutive entries in shared memory (a stored survivor comes from the
-//      head's own rows, at or behind its destination; a surviving new row from the caller's K/V),
-//      the cluster meets, and the run goes out with bulk stores.  The destinations of a round lie at
-//      or before its own cache sources and before those of every later round: in place.
+//      takes a run of consecutive entries out of memory (a stored survivor comes from the head's
+//      own rows, at or behind its destination; a surviving new row from the caller's K/V), most of
+//      them into shared memory, the rest into registers, the cluster meets, and the run goes out
+//      (bulk stores for the shared-memory part).  The destinations of a round lie at or before
+//      its own cache sources and before those of every later round: in place.
 //   7. heads that keep the whole new scale stop behind their stored survivors; the attention
 //      launch reads their new rows from the caller's tensors and appends them itself.
 //
@@ -58,9 +60,13 @@ constexpr int kMaxCpc = kTmemChunks - 1 + kMaxOver;      // 21 chunks = 2688 key
 constexpr int kMaxCluster = 8;
 constexpr uint32_t kCkDrainSpins = 1u << 22;
 constexpr int kMaxStages = 4;              // key tiles in flight per CTA (deeper rings measured no faster)
-constexpr int kMaxStageRows = 512;         // rows one CTA stages per round of the compaction
+constexpr int kHistBins = 4096;            // bins of a 12-bit digit of the radix select
+constexpr int kHistWords = kHistBins / 2;  // 16-bit counters, two per word
+constexpr int kMaxStageRows = 512;         // rows (K and V) in a CTA's staging buffers of the compaction
+constexpr int kMoveBuffers = 3;            // staging buffers of the compaction: loads run two rounds ahead of the stores
 constexpr size_t kSmemBudget = 227 * 1024; // dynamic shared memory a CTA may ask for
-static_assert(kCkThreads == 256, "one thread per histogram bin");
+static_assert(kHistBins == 16 * kCkThreads, "a thread sums 16 bins of the cluster's histograms");
+static_assert(kMaxCpc * kCkChunk < 65536, "16-bit counters per CTA");
 
 struct CkParams {
   int cluster;                // CTAs per head
@@ -68,7 +74,8 @@ struct CkParams {
   int n_over;                 // chunks of shared-memory logits reserved per CTA
   int tmem_cols;              // power of two >= 32
   int stages;                 // key tiles in the TMA ring (2 .. kMaxStages)
-  int stage_rows;             // rows (K and V) a CTA stages per round of the compaction
+  int region_bytes;           // front region of shared memory: ring, observation rows, overflow logits; later the row staging
+  int stage_rows;             // rows (K and V) a CTA stages in shared memory per round of the compaction
   int score_only;             // stop after the scores
   float* scores;              // [b*H, cand_stride] or nullptr
   int32_t* idx;               // [b*H, kept_stride]
@@ -86,11 +93,10 @@ struct CkShared {
   int pub_abort;                         // read by the other CTAs of the cluster
   float pub_stats[kMaxObs][2];           // this CTA's (max, sum-exp) per observation row
   int pub_counts[4];                     // kept above the threshold, equal to it; the same among stored candidates
-  int hist[2][256];
-  int tot[256];
+  int cnt_all[kMaxCluster][4];           // the counts of every CTA of the cluster
   float row_m[kMaxObs], row_inv_l[kMaxObs];
   int warp_sums[kCkThreads / 32 + 1];
-  int digit_of[kCkThreads / 32][2];      // per warp: the located digit and the rank left inside it
+  int digit_of[2][2];                    // the located digit, the rank left inside its bin, the bin's count
   int sh_abort;
   int cnt_old[2];
 };
@@ -102,6 +108,12 @@ __device__ __forceinline__ uint32_t cluster_rank() {
 }
 __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Execution barrier of the cluster without memory ordering: for a point that only has to come after
+// every CTA's loads have landed (nothing written before it is read by another CTA after it).
+__device__ __forceinline__ void cluster_sync_relaxed() {
+  __syncthreads();
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
 }
 // Address of the same shared-memory object in the CTA of rank `rank`.
 __device__ __forceinline__ uint32_t peer_addr(const void* p, uint32_t rank) {
@@ -119,6 +131,12 @@ __device__ __forceinline__ float ld_peer_f32(uint32_t addr) {
   asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
   return v;
 }
+__device__ __forceinline__ uint4 ld_peer_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared::cluster.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
 __device__ __forceinline__ void st_peer_i32(uint32_t addr, int v) {
   asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
@@ -128,7 +146,8 @@ __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ bool ck_wait(uint64_t* bar, uint32_t parity, CkShared* sh, int* status, int code,
                                         long long limit) {
@@ -156,6 +175,14 @@ __device__ __forceinline__ void ck_consumer_sync() { asm volatile("bar.sync 1, 1
 __device__ __forceinline__ uint32_t ck_orderable(float f) {
   const uint32_t u = __float_as_uint(f);
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// One more entry in bin `digit` of a histogram of 16-bit counters, two per word (a CTA holds fewer
+// than 65 536 keys).  Called by whole warps; lanes that fall into the same bin add once.
+__device__ __forceinline__ void hist_add(uint32_t* hist, bool in, uint32_t digit) {
+  const uint32_t peers = __match_any_sync(0xffffffffu, in ? digit : 0xffffffffu);
+  if (in && (threadIdx.x & 31) == __ffs(peers) - 1)
+    atomicAdd(&hist[digit >> 1], (uint32_t)__popc(peers) << (16 * (digit & 1)));
 }
 
 // Exclusive prefix sum of one value per thread over the CTA's kCkThreads threads, and the total.
@@ -188,30 +215,6 @@ __device__ __forceinline__ int ck_block_scan(int v, int* warp_sums, int& total) 
   return res;
 }
 
-// Warp 0 finds the digit d (from 255 down) at which the running count reaches `need`.
-__device__ __forceinline__ void ck_locate_digit(const int* hist, int need, int* sh_digit, int* sh_need) {
-  const int lane = threadIdx.x & 31;
-  int c[8];
-  int sum = 0;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) { c[i] = hist[255 - 8 * lane - i]; sum += c[i]; }
-  int incl = sum;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int n = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += n;
-  }
-  const int before = incl - sum;
-  if (before < need && need <= incl) {
-    int cum = before;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (cum < need && need <= cum + c[i]) { *sh_digit = 255 - 8 * lane - i; *sh_need = need - cum; }
-      cum += c[i];
-    }
-  }
-}
-
 template <int D>
 __global__ void __launch_bounds__(kCkThreads, 1)
 compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __grid_constant__ CUtensorMap tm_new,
@@ -225,10 +228,14 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
   const int STAGES = p.stages;
   const uint32_t RING_BYTES = (uint32_t)STAGES * K_BYTES;
 
-  pdl_wait();
+  // Nothing that another kernel writes is touched before pdl_wait() below: the head-type table is
+  // written when the cache is created, the step's lengths travel in the arguments.
   const int bh = blockIdx.y;
   const int ctx = a.is_ctx[bh % a.n_heads];
-  if (!a.trig[ctx]) return;                               // the whole cluster leaves together
+  if (!a.trig[ctx]) {                                     // the whole cluster leaves together
+    pdl_wait();
+    return;
+  }
   const int rank = (int)cluster_rank();
   const int CL = p.cluster;
   const int stored = a.stored[ctx], n_new = a.n_new, n_keep = a.kept[ctx];
@@ -248,12 +255,14 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
   const uint32_t k_sm = base;
   const uint32_t q_sm = base + RING_BYTES;
   float* over = reinterpret_cast<float*>(sm + RING_BYTES + SUB * Q_SUB_BYTES);            // [n_over][32][128]
-  uint32_t* keys = reinterpret_cast<uint32_t*>(over + (size_t)p.n_over * kMaxObs * kCkChunk);   // [cpc_max * 128]
-  int32_t* pos_stage = reinterpret_cast<int32_t*>(keys + (size_t)p.cpc_max * kCkChunk);        // [stage_rows]
-  int32_t* src_all = pos_stage + p.stage_rows;              // [cpc_max * 128 + stage_rows]: this CTA's list entries of every round
-  CkShared* sh = reinterpret_cast<CkShared*>(src_all + (size_t)p.cpc_max * kCkChunk + p.stage_rows);
+  const int S_ROWS = p.stage_rows;                          // rows a CTA holds in its staging buffers
+  uint32_t* keys = reinterpret_cast<uint32_t*>(sm + p.region_bytes);                            // [cpc_max * 128]
+  int32_t* pos_stage = reinterpret_cast<int32_t*>(keys + (size_t)p.cpc_max * kCkChunk);        // [S_ROWS]
+  int32_t* src_all = pos_stage + S_ROWS;                    // [cpc_max * 128 + S_ROWS]: this CTA's list entries of every round
+  CkShared* sh = reinterpret_cast<CkShared*>(src_all + (size_t)p.cpc_max * kCkChunk + S_ROWS);
   float* fold_m = reinterpret_cast<float*>(sm);           // [32][128], reuses the ring
   float* fold_l = fold_m + kMaxObs * kCkChunk;
+  uint32_t* hist32 = reinterpret_cast<uint32_t*>(sm);     // [2][kHistWords], reuses the ring after the fold
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -279,6 +288,15 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
     fence_barrier_init();
     fence_proxy_async();
   }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
+    tmem_relinquish();
+  }
+  if (warp == 0 && lane == 0) {
+    prefetch_tensormap(&tm_cache);
+    prefetch_tensormap(&tm_new);
+  }
+  pdl_wait();     // everything above overlaps the tail of the previous kernel
   // observation rows into the swizzled B tile; unused rows are zero
   for (int v = tid; v < kMaxObs * (D / 8); v += kCkThreads) {
     const int i = v / (D / 8), c = v % (D / 8);
@@ -291,10 +309,6 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
     *reinterpret_cast<uint4*>(sm + RING_BYTES + off) = val;
   }
   fence_proxy_async();
-  if (warp == 1) {
-    tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
-    tmem_relinquish();
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -306,8 +320,6 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
   const uint32_t t_lane = tmem + (static_cast<uint32_t>(quad * 32) << 16);
   if (warp == 0) {
     if (lane == 0) {
-      prefetch_tensormap(&tm_cache);
-      prefetch_tensormap(&tm_new);
       int issued = 0;
       bool ok = true;
       for (int i = 0; i < n_run; ++i) {
@@ -421,6 +433,12 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
   }
   __syncthreads();
   if (tid == 0) sh->pub_abort = *reinterpret_cast<volatile int*>(&sh->abort_flag);
+  // the ring is idle from here on; its first 16 KB become the two histograms of the radix select
+  {
+    uint4* z = reinterpret_cast<uint4*>(hist32 + 8 * tid);
+    z[0] = z[1] = make_uint4(0, 0, 0, 0);
+    z[kHistWords / 4] = z[kHistWords / 4 + 1] = make_uint4(0, 0, 0, 0);
+  }
 
   // ------------------------------------------------------------------ 2. row statistics of the whole head
   cluster_sync();
@@ -428,9 +446,11 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
     float mr[kMaxCluster], lr[kMaxCluster];
 #pragma unroll
     for (int r = 0; r < kMaxCluster; ++r) {                 // all loads in flight at once
-      const int rr = r < CL ? r : 0;
-      mr[r] = ld_peer_f32(peer_addr(&sh->pub_stats[tid][0], rr));
-      lr[r] = ld_peer_f32(peer_addr(&sh->pub_stats[tid][1], rr));
+      mr[r] = lr[r] = 0.f;
+      if (r < CL) {
+        mr[r] = ld_peer_f32(peer_addr(&sh->pub_stats[tid][0], r));
+        lr[r] = ld_peer_f32(peer_addr(&sh->pub_stats[tid][1], r));
+      }
     }
     float m = -INFINITY;
 #pragma unroll
@@ -464,7 +484,9 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
       // a chunk of protected candidates only (the new scale of a structural head) is kept whatever
       // its scores are; they are formed only when the caller wants them
       if (!p.scores && structural && a.protect_new && c_begin + i >= n_sc) {
+        int j;
         keys[i * kCkChunk + key_row] = 0xffffffffu;
+        hist_add(hist32, slot_info(i * kCkChunk + key_row, j), kHistBins - 1);
         continue;
       }
       uint32_t acc[kMaxObs];
@@ -492,6 +514,7 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
         }
       }
       keys[i * kCkChunk + key_row] = key;
+      if (!p.score_only) hist_add(hist32, live, key >> 20);   // first digit of the radix select
     }
   }
   tc_fence_before();
@@ -499,51 +522,85 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
 
   if (!aborted && !p.score_only) {
     // ---------------------------------------------------------------- 4. radix select over the cluster
+    // Digits of 12, 12 and 8 bits.  The local histogram of the first digit was filled while the keys
+    // were formed; the select stops as soon as every entry left in the located bin survives, which
+    // with 24 bits fixed is the usual case.
     const int n_slots = cpc * kCkChunk;
     uint32_t prefix = 0, mask = 0;
     int need = n_keep;
-    sh->hist[0][tid] = 0;                                     // kCkThreads == 256 bins
-    sh->hist[1][tid] = 0;
-    __syncthreads();
 #pragma unroll 1
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      int* hist = sh->hist[pass & 1];
-      for (int s0 = 0; s0 < n_slots; s0 += kCkThreads) {
-        const int slot = s0 + tid;
-        int j;
-        const bool live = slot < n_slots && slot_info(slot, j);
-        const uint32_t k = live ? keys[slot] : 0u;
-        const bool in = live && ((k & mask) == prefix);
-        const uint32_t digit = in ? ((k >> shift) & 255u) : 256u;
-        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-        if (in && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+    for (int pass = 0; pass < 3; ++pass) {
+      const int shift = pass == 0 ? 20 : (pass == 1 ? 8 : 0);
+      const uint32_t dmask = pass == 2 ? 255u : 4095u;
+      uint32_t* hist = hist32 + (pass & 1) * kHistWords;
+      if (pass > 0) {
+        for (int s0 = 0; s0 < n_slots; s0 += kCkThreads) {
+          const int slot = s0 + tid;
+          int j;
+          const bool live = slot < n_slots && slot_info(slot, j);
+          const uint32_t k = live ? keys[slot] : 0u;
+          const bool in = live && ((k & mask) == prefix);
+          hist_add(hist, in, (k >> shift) & dmask);
+        }
       }
-      __syncthreads();
-      cluster_sync();
-      {
-        int part[kMaxCluster];
+      cluster_sync();                                         // (orders the CTA's own threads as well)
+      // thread t owns bins [16 t, 16 t + 16): two 16-bit counters per word
+      int c[16];
 #pragma unroll
-        for (int r = 0; r < kMaxCluster; ++r) part[r] = ld_peer_i32(peer_addr(&hist[tid], r < CL ? r : 0));
-        int t = 0;
+      for (int i = 0; i < 16; ++i) c[i] = 0;
+      {
+        uint4 part[kMaxCluster][2];
+#pragma unroll
+        for (int r = 0; r < kMaxCluster; ++r)                 // all loads in flight at once
+          if (r < CL && (pass < 2 || tid < 16)) {               // the 8-bit digit fills 256 bins only
+            const uint32_t addr = peer_addr(hist + 8 * tid, r);
+            part[r][0] = ld_peer_v4(addr);
+            part[r][1] = ld_peer_v4(addr + 16);
+          } else {
+            part[r][0] = part[r][1] = make_uint4(0, 0, 0, 0);
+          }
 #pragma unroll
         for (int r = 0; r < kMaxCluster; ++r)
-          if (r < CL) t += part[r];
-        sh->tot[tid] = t;
+          if (r < CL) {
+            const uint32_t w[8] = {part[r][0].x, part[r][0].y, part[r][0].z, part[r][0].w,
+                                   part[r][1].x, part[r][1].y, part[r][1].z, part[r][1].w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { c[2 * i] += (int)(w[i] & 0xffffu); c[2 * i + 1] += (int)(w[i] >> 16); }
+          }
       }
       // the other buffer is free: every CTA read it before it arrived at the barrier above
-      sh->hist[(pass & 1) ^ 1][tid] = 0;
+      {
+        uint4* z = reinterpret_cast<uint4*>(hist32 + ((pass & 1) ^ 1) * kHistWords + 8 * tid);
+        z[0] = make_uint4(0, 0, 0, 0);
+        z[1] = make_uint4(0, 0, 0, 0);
+      }
+      int mine = 0;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) mine += c[i];
+      int total;
+      const int below = ck_block_scan(mine, sh->warp_sums, total);
+      const int above = total - below - mine;                 // entries in the bins of the threads behind this one
+      if (above < need && need <= above + mine) {
+        int cum = above;
+#pragma unroll
+        for (int i = 15; i >= 0; --i) {
+          if (cum < need && need <= cum + c[i]) {
+            sh->digit_of[0][0] = 16 * tid + i;
+            sh->digit_of[0][1] = need - cum;
+            sh->digit_of[1][0] = c[i];
+          }
+          cum += c[i];
+        }
+      }
       __syncthreads();
-      // every warp locates the digit for itself (same totals, same result); lane 0 of warp w
-      // leaves it in a slot of its own
-      ck_locate_digit(sh->tot, need, &sh->digit_of[warp][0], &sh->digit_of[warp][1]);
-      __syncwarp();
-      prefix |= (uint32_t)sh->digit_of[warp][0] << shift;
-      need = sh->digit_of[warp][1];
-      mask |= 255u << shift;
+      prefix |= (uint32_t)sh->digit_of[0][0] << shift;
+      need = sh->digit_of[0][1];
+      mask |= dmask << shift;
+      if (need == sh->digit_of[1][0]) break;                  // the same in every CTA of the cluster
     }
     // ---------------------------------------------------------------- 5. ascending index list
-    // prefix = key of the n_keep-th largest entry; `need` of the entries equal to it survive (lowest indices)
+    // prefix = the fixed digits of the n_keep-th largest key; of the entries that agree with it in
+    // those digits `need` survive (lowest indices; all of them when the select stopped early)
     const uint32_t thr = prefix;
     const int per = (n_slots + kCkThreads - 1) / kCkThreads;  // thread t owns slots [t*per, t*per + per)
     int gt = 0, eq = 0, gt_old = 0, eq_old = 0;
@@ -551,7 +608,7 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
       const int slot = tid * per + e;
       int j;
       if (slot < n_slots && slot_info(slot, j)) {
-        const uint32_t k = keys[slot];
+        const uint32_t k = keys[slot] & mask;
         gt += k > thr;
         eq += k == thr;
         if (j < stored) { gt_old += k > thr; eq_old += k == thr; }
@@ -567,24 +624,19 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
       sh->pub_counts[2] = sh->cnt_old[0];
       sh->pub_counts[3] = sh->cnt_old[1];
     }
-    __syncthreads();
     cluster_sync();
     int gt_before = packed & 0xffff, eq_before = packed >> 16;
     int gt_old_all = 0, eq_old_all = 0;
-    {
-      int cnt[kMaxCluster][4];
+    // one remote load per count, then every thread reads the CTA's own copy
+    if (tid < 4 * CL) sh->cnt_all[tid >> 2][tid & 3] = ld_peer_i32(peer_addr(&sh->pub_counts[tid & 3], tid >> 2));
+    __syncthreads();
 #pragma unroll
-      for (int r = 0; r < kMaxCluster; ++r)
-#pragma unroll
-        for (int x = 0; x < 4; ++x) cnt[r][x] = ld_peer_i32(peer_addr(&sh->pub_counts[x], r < CL ? r : 0));
-#pragma unroll
-      for (int r = 0; r < kMaxCluster; ++r)
-        if (r < CL) {
-          if (r < rank) { gt_before += cnt[r][0]; eq_before += cnt[r][1]; }
-          gt_old_all += cnt[r][2];
-          eq_old_all += cnt[r][3];
-        }
-    }
+    for (int r = 0; r < kMaxCluster; ++r)
+      if (r < CL) {
+        if (r < rank) { gt_before += sh->cnt_all[r][0]; eq_before += sh->cnt_all[r][1]; }
+        gt_old_all += sh->cnt_all[r][2];
+        eq_old_all += sh->cnt_all[r][3];
+      }
     const int n_old = gt_old_all + min(eq_old_all, need);     // survivors that were already stored
     // Entry o of the head's ascending list is candidate j.  Entry o becomes row o of the head, and
     // rows are compacted in rounds of CL * S consecutive entries, CTA `rk` of the cluster staging S
@@ -592,7 +644,10 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
     // scale need only their stored survivors (the attention launch appends the rest).
     const bool attend_appends = a.seg_new[ctx] != 0;
     const int n_rows = attend_appends ? n_old : n_keep;
-    const int S = p.stage_rows, RS = CL * S;
+    // rounds: as few as the staging buffers (a third of the staging rows each) allow, of equal size
+    const int s_cap = S_ROWS / kMoveBuffers;
+    const int n_rounds = (n_rows + CL * s_cap - 1) / (CL * s_cap);
+    const int S = n_rounds > 0 ? (n_rows + CL * n_rounds - 1) / (CL * n_rounds) : 1, RS = CL * S;
     auto deliver = [&](int o, int j) {
       if (o < n_rows && dbg_ok(o >= 0 && o < n_keep, a.status, 9)) {
         const int t = o / RS, w = o - t * RS, rk = w / S, lr = w - rk * S;
@@ -603,7 +658,7 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
       const int slot = tid * per + e;
       int j;
       if (slot < n_slots && slot_info(slot, j)) {
-        const uint32_t k = keys[slot];
+        const uint32_t k = keys[slot] & mask;
         if (k > thr) {
           deliver(gt_before + min(eq_before, need), j);
           ++gt_before;
@@ -613,7 +668,6 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
         }
       }
     }
-    __syncthreads();
     cluster_sync();                                           // every CTA holds its part of the list
 
     // ---------------------------------------------------------------- 6. and 7. compaction in rounds
@@ -630,53 +684,72 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
     const uint4* kn = p.k_new + (size_t)bh * n_new * PIECES;
     const uint4* vn = p.v_new + (size_t)bh * n_new * PIECES;
     constexpr uint32_t ROWB = PIECES * 16;
-    const uint32_t v_base = base + (uint32_t)S * ROWB;       // staging: S key rows, then S value rows
-    int t = 0;
-    for (int r0 = 0; r0 < n_rows; r0 += RS, ++t) {
-      const int first = r0 + rank * S;
-      const int rows = max(0, min(S, n_rows - first));
-      const int32_t* srcs = src_all + t * S;
-      // ascending entries with source >= destination: if the last stored row of the slice stays
-      // where it is, so does every row of the slice
-      const bool moving = rows > 0 && !(srcs[rows - 1] == first + rows - 1 && srcs[rows - 1] < stored);
-      if (moving) {
+    // Staging buffer b holds S key rows, then S value rows.  The loads of round t + 2 are issued
+    // while round t stores: a later round's sources lie behind every earlier round's destinations.
+    const uint32_t buf_bytes = 2u * (uint32_t)s_cap * ROWB;
+    auto slice_first = [&](int t) { return t * RS + rank * S; };
+    auto slice_rows = [&](int t) { return max(0, min(S, n_rows - slice_first(t))); };
+    // ascending entries with source >= destination: if the last stored row of the slice stays
+    // where it is, so does every row of the slice
+    auto slice_moves = [&](int t) {
+      const int rows = slice_rows(t), last = src_all[t * S + max(rows, 1) - 1];
+      return rows > 0 && !(last == slice_first(t) + rows - 1 && last < stored);
+    };
+    auto issue_loads = [&](int t) {
+      if (t < n_rounds && slice_moves(t)) {
+        const int first = slice_first(t), rows = slice_rows(t);
+        const int32_t* srcs = src_all + t * S;
+        const uint32_t kb = base + (uint32_t)(t % kMoveBuffers) * buf_bytes, vb = kb + (uint32_t)S * ROWB;
+        int32_t* ps = pos_stage + (t % kMoveBuffers) * s_cap;
         for (int v = tid; v < rows * PIECES; v += kCkThreads) {
           const int lr = v / PIECES, piece = v % PIECES;
           int src = srcs[lr];
           // a checked build turns an entry outside [destination, candidates) into "stays where it is"
-          if (!dbg_ok(src >= first + lr && src < stored + n_new && first + lr < a.cap[ctx], a.status, 10)) src = first + lr < stored ? first + lr : stored;
+          if (!dbg_ok(src >= first + lr && src < stored + n_new && first + lr < a.cap[ctx], a.status, 10))
+            src = first + lr < stored ? first + lr : stored;
           const uint4* ks = src < stored ? kp + (size_t)src * PIECES : kn + (size_t)(src - stored) * PIECES;
           const uint4* vs = src < stored ? vp + (size_t)src * PIECES : vn + (size_t)(src - stored) * PIECES;
-          cp_async16(base + (uint32_t)lr * ROWB + piece * 16, ks + piece);
-          cp_async16(v_base + (uint32_t)lr * ROWB + piece * 16, vs + piece);
+          cp_async16(kb + (uint32_t)lr * ROWB + piece * 16, ks + piece);
+          cp_async16(vb + (uint32_t)lr * ROWB + piece * 16, vs + piece);
         }
         for (int lr = tid; lr < rows; lr += kCkThreads) {
           const int src = srcs[lr];
-          if (src < stored) cp_async4(smem_u32(&pos_stage[lr]), pos + max(src, 0));
-          else pos_stage[lr] = a.pos_base + (src - stored);
+          if (src < stored) cp_async4(smem_u32(&ps[lr]), pos + max(src, 0));
+          else ps[lr] = a.pos_base + (src - stored);
         }
-        cp_async_wait_all();
-        fence_proxy_async();                                  // the bulk stores below read what these threads wrote
       }
-      __syncthreads();
-      cluster_sync();                                         // every source of this round has been read
+      cp_async_commit();                                      // one group per round, empty or not
+    };
+    issue_loads(0);
+    issue_loads(1);
+    for (int t = 0; t < n_rounds; ++t) {
+      cp_async_wait_group<1>();                               // the loads of round t (all but the latest group) have landed
+      fence_proxy_async();                                    // the bulk stores below read what these threads wrote
+      cluster_sync_relaxed();                                 // every source of this round has been read
+      const bool moving = slice_moves(t);
       if (moving) {
+        const int first = slice_first(t), rows = slice_rows(t);
+        const uint32_t kb = base + (uint32_t)(t % kMoveBuffers) * buf_bytes, vb = kb + (uint32_t)S * ROWB;
         if (tid == 0) {
           constexpr uint32_t kPiece = 32768;                  // bytes per bulk store
           const uint32_t bytes = (uint32_t)rows * ROWB;
           for (uint32_t o = 0; o < bytes; o += kPiece) {
             const uint32_t n = min(kPiece, bytes - o);
-            bulk_store(reinterpret_cast<unsigned char*>(kp + (size_t)first * PIECES) + o, base + o, n);
-            bulk_store(reinterpret_cast<unsigned char*>(vp + (size_t)first * PIECES) + o, v_base + o, n);
+            bulk_store(reinterpret_cast<unsigned char*>(kp + (size_t)first * PIECES) + o, kb + o, n);
+            bulk_store(reinterpret_cast<unsigned char*>(vp + (size_t)first * PIECES) + o, vb + o, n);
           }
-          bulk_commit();
         }
-        for (int lr = tid; lr < rows; lr += kCkThreads) pos[first + lr] = pos_stage[lr];
-        if (tid == 0) bulk_wait_read<0>();                    // the staging area is reused by the next round
+        const int32_t* ps = pos_stage + (t % kMoveBuffers) * s_cap;
+        for (int lr = tid; lr < rows; lr += kCkThreads) pos[first + lr] = ps[lr];
+      }
+      if (tid == 0) {
+        bulk_commit();                                        // one group per round, empty or not
+        bulk_wait_read<1>();                                  // round t - 1 has left its buffer, which round t + 2 fills
       }
       __syncthreads();
+      issue_loads(t + 2);
     }
-    if (tid == 0) bulk_wait<0>();                             // the rows are in place before the CTA leaves
+    if (tid == 0) bulk_wait_read<0>();                        // shared memory is read out before the CTA leaves
   }
   // no CTA leaves while another may still read its shared memory
   cluster_sync();
@@ -686,29 +759,34 @@ compress_cluster_kernel(const __grid_constant__ CUtensorMap tm_cache, const __gr
   }
 }
 
-// Shared memory of one CTA: ring, observation rows and overflow logits (the compaction later
-// stages rows over all three), keys, the two per-row staging arrays, barriers and exchange area.
+// Shared memory of one CTA: the front region (ring, observation rows and overflow logits; the
+// compaction later stages rows over all of it), keys, the two per-row staging arrays, barriers and
+// exchange area.
 template <int D>
 size_t ck_smem_bytes(const CkParams& p) {
-  return 1024 + (size_t)p.stages * (D / 64) * kCkChunk * 128 + (size_t)(D / 64) * kMaxObs * 128 +
-         (size_t)p.n_over * kMaxObs * kCkChunk * sizeof(float) + (size_t)p.cpc_max * kCkChunk * sizeof(uint32_t) +
-         (2 * (size_t)p.stage_rows + (size_t)p.cpc_max * kCkChunk) * sizeof(int32_t) + sizeof(CkShared) + 64;
+  const size_t rows = (size_t)p.stage_rows;
+  return 1024 + (size_t)p.region_bytes + (size_t)p.cpc_max * kCkChunk * sizeof(uint32_t) +
+         (2 * rows + (size_t)p.cpc_max * kCkChunk) * sizeof(int32_t) + sizeof(CkShared) + 64;
 }
 
 // Ring depth and staging rows for this launch: as many key tiles in flight as the CTA has chunks
-// (more would never be used) and as shared memory holds; the compaction stages rows over the
-// ring, the observation rows and the overflow logits.
+// (more would never be used) and as shared memory holds; the front region then grows to what is
+// left of the budget, so that a round of the compaction stages as many rows as possible.
 template <int D>
 void ck_size(CkParams& p) {
   const size_t k_bytes = (size_t)(D / 64) * kCkChunk * 128;
-  p.stages = 2;
+  const size_t row_bytes = 2 * (size_t)D * 2;                // a key row and a value row
+  const size_t q_over = (size_t)(D / 64) * kMaxObs * 128 + (size_t)p.n_over * kMaxObs * kCkChunk * sizeof(float);
   p.stage_rows = kMaxStageRows;
-  const size_t fixed = ck_smem_bytes<D>(p) - 2 * k_bytes;
-  int fit = (int)((kSmemBudget - fixed) / k_bytes);
+  p.region_bytes = 0;
+  const size_t other = ck_smem_bytes<D>(p);                   // everything but the front region
+  const size_t room = kSmemBudget > other ? kSmemBudget - other : 0;
+  const int fit = room > q_over ? (int)((room - q_over) / k_bytes) : 0;
   p.stages = std::max(2, std::min({fit, kMaxStages, std::max(p.cpc_max, 2)}));
-  const size_t stage_bytes = p.stages * k_bytes + (size_t)(D / 64) * kMaxObs * 128 +
-                             (size_t)p.n_over * kMaxObs * kCkChunk * sizeof(float);
-  p.stage_rows = (int)std::min<size_t>(kMaxStageRows, stage_bytes / (2 * (size_t)D * 2));
+  const size_t need = p.stages * k_bytes + q_over;
+  const size_t region = std::max(need, std::min(room, (size_t)kMaxStageRows * row_bytes)) / 1024 * 1024;
+  p.region_bytes = (int)std::max(region, (need + 1023) / 1024 * 1024);
+  p.stage_rows = (int)std::min<size_t>(kMaxStageRows, p.region_bytes / row_bytes);
 }
 
 template <int D>

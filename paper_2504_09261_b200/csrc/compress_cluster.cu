@@ -833,7 +833,7 @@ int ck_active_clusters(const StepArgs& a, const CkParams& p) {
 
 template <int D>
 int launch_t(const StepArgs& a, const CUtensorMap& tm_cache, const CUtensorMap& tm_new, const void* q, CkParams p,
-             int max_chunks, int n_clusters, cudaStream_t st) {
+             int max_chunks, int n_clusters, int reserved_sms, cudaStream_t st) {
   // the opt-in is made once per (kernel, device), so it asks for the most any launch can need
   if (!allow_dynamic_smem(compress_cluster_kernel<D>, kSmemBudget)) return -1;
   // CTAs per head: at least what holds the longest candidate list; more spread the key stream over
@@ -849,7 +849,11 @@ int launch_t(const StepArgs& a, const CUtensorMap& tm_cache, const CUtensorMap& 
   };
   int cl = p.cluster;
   shape(cl);
+  // a launch that runs beside another one leaves that one its SMs, if both fit the device at all
+  const int sms = sm_count();
+  const bool beside = reserved_sms > 0 && n_clusters * cl + reserved_sms <= sms;
   while (cl < kMaxCluster && (max_chunks + 2 * cl - 1) / (2 * cl) >= 2) {
+    if (beside && n_clusters * 2 * cl + reserved_sms > sms) break;
     shape(2 * cl);
     if (ck_active_clusters<D>(a, p) < n_clusters) break;
     cl *= 2;
@@ -870,9 +874,10 @@ int launch_t(const StepArgs& a, const CUtensorMap& tm_cache, const CUtensorMap& 
 // Scores only (scores != nullptr, idx == nullptr) or the whole compression of the step (idx != nullptr).
 // Returns 1 (one launch), -1 on a launch error, or 0 when this step is outside what the kernel holds
 // (candidate lists beyond 8 x 21 chunks per head, the every-query scoring rounds): the caller then
-// takes the separate scoring, selection and compaction launches.
+// takes the separate scoring, selection and compaction launches.  reserved_sms: CTAs of a launch
+// that is enqueued to run beside this one (0 if none).
 int launch_compress_cluster(const StepArgs& a, const void* q, const void* k_new, const void* v_new, float* scores,
-                            int32_t* idx, cudaStream_t st) {
+                            int32_t* idx, cudaStream_t st, int reserved_sms) {
   if (!a.k_map || a.obs_full || a.score_accumulate) return 0;
   int max_chunks = 0, types = 0;
   const int n_new_chunks = (a.n_new + kCkChunk - 1) / kCkChunk;
@@ -901,8 +906,8 @@ int launch_compress_cluster(const StepArgs& a, const void* q, const void* k_new,
     return -1;
   }
   const CUtensorMap& tm_cache = *static_cast<const CUtensorMap*>(a.k_map);
-  return a.head_dim == 128 ? launch_t<128>(a, tm_cache, tm_new, q, p, max_chunks, n_clusters, st)
-                           : launch_t<64>(a, tm_cache, tm_new, q, p, max_chunks, n_clusters, st);
+  return a.head_dim == 128 ? launch_t<128>(a, tm_cache, tm_new, q, p, max_chunks, n_clusters, reserved_sms, st)
+                           : launch_t<64>(a, tm_cache, tm_new, q, p, max_chunks, n_clusters, reserved_sms, st);
 }
 
 }  // namespace hack

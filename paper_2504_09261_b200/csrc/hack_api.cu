@@ -831,7 +831,9 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
   if (any && fused_append) {
     // score, select and compact in one cluster launch per head (counted with the scoring stage)
     StageScope ts(c, st, 0);
-    if ((r = hack::launch_compress_cluster(a, q, k, v, nullptr, c->idx, st)) < 0) return HACK_ERR_CUDA;
+    // the appending heads' attention (two query tiles per CTA) runs beside this launch
+    const int beside = can_fork ? n_heads_of[1 - trig_type] * ((p.n_new + 255) / 256) : 0;
+    if ((r = hack::launch_compress_cluster(a, q, k, v, nullptr, c->idx, st, beside)) < 0) return HACK_ERR_CUDA;
     ts.done(r);
     n += r;
     compressed = r > 0;

@@ -87,7 +87,7 @@ int launch_select(const StepArgs& a, const float* scores, int32_t* idx, int32_t*
 // in one launch of one thread-block cluster per head.  1: launched; 0: the step is outside what the
 // kernel holds, take the separate launches; -1: launch error.
 int launch_compress_cluster(const StepArgs& a, const void* q, const void* k_new, const void* v_new, float* scores,
-                            int32_t* idx, cudaStream_t st);
+                            int32_t* idx, cudaStream_t st, int reserved_sms = 0);
 // idx == nullptr: every head appends (keeps all candidates).  idx_all != 0: idx rows are valid for
 // heads that are not triggered as well (identity lists written by launch_select).
 int launch_compact(const StepArgs& a, int dtype, const int32_t* idx, int idx_all, const void* k_new,

@@ -125,7 +125,8 @@ template <int D>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kn,
-                 const __grid_constant__ CUtensorMap tm_vn, const TcParams p) {
+                 const __grid_constant__ CUtensorMap tm_vn, const __grid_constant__ CUtensorMap tm_o,
+                 const TcParams p) {
   constexpr int SUB = D / 64;                       // 64-column (128-byte) sub-tiles per row
   constexpr uint32_t SUB_BYTES = kBN * 128;         // one sub-tile: 128 rows x 128 bytes
   constexpr uint32_t TILE_BYTES = SUB * SUB_BYTES;
@@ -182,6 +183,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     prefetch_tensormap(&tm_q);
     prefetch_tensormap(&tm_k);
     prefetch_tensormap(&tm_v);
+    prefetch_tensormap(&tm_o);
     if (len_b > 0) {
       prefetch_tensormap(&tm_kn);
       prefetch_tensormap(&tm_vn);
@@ -480,31 +482,48 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[t]));
       }
       if (ok) ok = __all_sync(0xffffffffu, wait_bar(&bars->o_final[t], 0, bars, p.status, 9, wlim));
-      if (ok) {
+      // the four warps of the tile meet on a named barrier below, so they agree first on whether all of them got here
+      uint32_t all_ok;
+      asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                   : "=r"(all_ok) : "r"((uint32_t)ok), "r"(1 + t) : "memory");
+      if (all_ok) {
         tc_fence_after();
         const int row = q0 + t * kBM + r;
         const float inv = 1.f / l;
-        __nv_bfloat16* dst = p.out + (static_cast<size_t>(bh) * p.n_new + row) * D;
         if (p.row_stats && row < p.n_new)
           *reinterpret_cast<float2*>(p.row_stats + (static_cast<size_t>(bh) * p.n_new + row) * 2) = make_float2(m_used, l);
+        // The tile's output goes through its query tile's shared memory (the last Q K^T product has
+        // read it), laid out as a tiled copy with the 128-byte swizzle expects it: thread r's 16-byte
+        // pieces of a store instruction fall into different banks, and one tiled store per 64
+        // columns writes whole rows (a thread storing its own row straight to memory wrote 32
+        // half-used sectors per instruction: 3 us per CTA against 1).  Rows past the head's last
+        // query lie outside the tensor and are not written.
+        const uint32_t o_sm = q_sm + t * TILE_BYTES + r * 128;
 #pragma unroll
         for (int ch = 0; ch < D / 32; ++ch) {
           uint32_t orr[32];
           tmem_ld32(o_addr + ch * 32, orr);
           tmem_wait_ld();
-          if (row < p.n_new) {
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint32_t w[4];
+          for (int v = 0; v < 4; ++v) {
+            uint32_t w[4];
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(orr[v * 8 + 2 * e]) * inv,
-                                                                __uint_as_float(orr[v * 8 + 2 * e + 1]) * inv);
-                w[e] = *reinterpret_cast<const uint32_t*>(&hh);
-              }
-              *reinterpret_cast<uint4*>(dst + ch * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            for (int e = 0; e < 4; ++e) {
+              const __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(orr[v * 8 + 2 * e]) * inv,
+                                                              __uint_as_float(orr[v * 8 + 2 * e + 1]) * inv);
+              w[e] = *reinterpret_cast<const uint32_t*>(&hh);
             }
+            const int piece = ch * 4 + v;                      // 16-byte piece of the row
+            st_shared_v4(o_sm + (piece >> 3) * SUB_BYTES + (((piece & 7) ^ (r & 7)) << 4), w[0], w[1], w[2], w[3]);
           }
+        }
+        fence_proxy_async();                                   // the tiled store reads what these threads wrote
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
+        if (r == 0) {
+#pragma unroll
+          for (int cc = 0; cc < SUB; ++cc) tma_store_3d(&tm_o, cc * 64, q0 + t * kBM, bh, q_sm + t * TILE_BYTES + cc * SUB_BYTES);
+          bulk_commit();
+          bulk_wait_read<0>();                                 // shared memory is read out before the CTA leaves
         }
       }
     }
@@ -553,12 +572,33 @@ bool make_rows_map(void* out_map, const void* base, uint64_t rows, int head_dim)
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+namespace {
+// 3-D bf16 tensor map over the output [heads, n_new, head_dim] (boxes of 128 rows x 64 columns of one
+// head, 128-byte swizzle): a tile that reaches past the head's last query row is clipped there.
+bool make_out_map(CUtensorMap* out_map, const void* base, int heads, int n_new, int head_dim) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || heads <= 0 || n_new <= 0) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_new, (cuuint64_t)heads};
+  const cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)n_new * head_dim * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)kBM, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(out_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+}  // namespace
+
 int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
                      const void* q, void* out, float* row_stats, const void* k_new, const void* v_new,
                      int n_heads_served, bool shares_gpu, cudaStream_t st) {
   CUtensorMap tm_q;
   if (!make_rows_map(&tm_q, q, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) {
     set_error("attention: cuTensorMapEncodeTiled failed for the queries");
+    return -1;
+  }
+  CUtensorMap tm_o;
+  if (!make_out_map(&tm_o, out, a.batch * a.n_heads, a.n_new, a.head_dim)) {
+    set_error("attention: cuTensorMapEncodeTiled failed for the output");
     return -1;
   }
   TcParams p;
@@ -608,11 +648,11 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
   const int grid = p.n_pairs * heads;
   if (a.head_dim == 128) {
     if (!allow_dynamic_smem(attend_tc_kernel<128>, tc_smem_bytes<128>())) return -1;
-    launch_k(attend_tc_kernel<128>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, tm_kn, tm_vn, p);
+    launch_k(attend_tc_kernel<128>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, tm_kn, tm_vn, tm_o, p);
   } else {
     if (!allow_dynamic_smem(attend_tc_kernel<64>, tc_smem_bytes<128>())) return -1;
     // the larger request keeps it at one CTA per SM (the kernel owns all 512 TMEM columns)
-    launch_k(attend_tc_kernel<64>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, tm_kn, tm_vn, p);
+    launch_k(attend_tc_kernel<64>, grid, kThreadsTc, tc_smem_bytes<128>(), st, tm_q, tk, tv, tm_kn, tm_vn, tm_o, p);
   }
   return launched(1);
 }

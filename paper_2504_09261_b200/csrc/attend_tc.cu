@@ -46,6 +46,9 @@
 // is protected, Eq. 11) are served that way before the new rows are in the cache: the append
 // (Eq. 3) is done by warp 3 of the same CTAs with bulk copies through a small staging buffer, each
 // CTA of a head taking a slice of the rows; nothing in this launch reads the rows they write.
+// A tile's output rows leave through the shared memory of its query tile (free once the last Q K^T
+// product has read it) and one tiled store per 64 columns; the store's 3-D tensor map of the output
+// clips the rows behind a head's last query.
 // Every mbarrier wait is bounded; on expiry the CTA raises the status word, drains what it has in
 // flight, frees its TMEM and returns.
 #include <cuda.h>

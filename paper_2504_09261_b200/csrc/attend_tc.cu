@@ -78,6 +78,7 @@ struct TcParams {
   int tiles_per_cta;                     // 2, or 1 when the grid would not fill the GPU otherwise
   int len_a[2], len_b[2];                // per head type: rows read from the cache, then from the caller's K/V
   int append_new;                        // heads with len_b > 0 also store those rows behind their len_a cache rows
+  int q_before_wait;                     // the queries may be read ahead of the dependency wait
   int pos_base;                          // global position of the new scale's first token
   int head_dim_pieces;                   // 16-byte pieces per row
   int cap[2];                            // rows a head of each type owns (checked builds)
@@ -191,13 +192,21 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       prefetch_tensormap(&tm_kn);
       prefetch_tensormap(&tm_vn);
     }
+    // The queries are the caller's input.  When the kernel ahead of this one in the stream is the
+    // step's own compression launch, whatever produced them had completed before that launch passed
+    // its dependency wait, hence before any CTA of this launch started: they are loaded ahead of the
+    // wait, under the compression's last CTAs.
+    auto load_queries = [&]() {
+      for (int t = 0; t < ntile; ++t) {
+        const uint32_t bar = smem_u32(&bars->q_full[t]);
+        mbar_expect_tx(bar, TILE_BYTES);
+        for (int c = 0; c < SUB; ++c)
+          tma_load_2d(q_sm + t * TILE_BYTES + c * SUB_BYTES, &tm_q, c * 64, qrow + t * kBM, bar);
+      }
+    };
+    if (p.q_before_wait) load_queries();
     pdl_wait();
-    for (int t = 0; t < ntile; ++t) {
-      const uint32_t bar = smem_u32(&bars->q_full[t]);
-      mbar_expect_tx(bar, TILE_BYTES);
-      for (int c = 0; c < SUB; ++c)
-        tma_load_2d(q_sm + t * TILE_BYTES + c * SUB_BYTES, &tm_q, c * 64, qrow + t * kBM, bar);
-    }
+    if (!p.q_before_wait) load_queries();
     mbar_expect_tx(smem_u32(&bars->k_full[0]), TILE_BYTES);
     for (int c = 0; c < SUB; ++c) tma_load_2d(k_sm + c * SUB_BYTES, k_src(0), c * 64, tile_row(0), smem_u32(&bars->k_full[0]));
     mbar_expect_tx(smem_u32(&bars->v_full[0]), TILE_BYTES);
@@ -593,7 +602,7 @@ bool make_out_map(CUtensorMap* out_map, const void* base, int heads, int n_new, 
 
 int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
                      const void* q, void* out, float* row_stats, const void* k_new, const void* v_new,
-                     int n_heads_served, bool shares_gpu, cudaStream_t st) {
+                     int n_heads_served, bool shares_gpu, cudaStream_t st, bool follows_compression) {
   CUtensorMap tm_q;
   if (!make_rows_map(&tm_q, q, (uint64_t)a.batch * a.n_heads * a.n_new, a.head_dim)) {
     set_error("attention: cuTensorMapEncodeTiled failed for the queries");
@@ -631,6 +640,7 @@ int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, co
       return -1;
     }
   }
+  p.q_before_wait = follows_compression ? 1 : 0;
   p.pos_base = a.pos_base;
   p.head_dim_pieces = a.head_dim * 2 / 16;
   p.cap[0] = a.cap[0];

@@ -693,7 +693,7 @@ hack_status_t hack_compact(hack_cache_t* c, int32_t layer, int32_t scale, const 
 static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void* q, void* out, float* sigma,
                                  cudaStream_t st, const void* k_new = nullptr, const void* v_new = nullptr,
                                  const int* seg_new = nullptr, int only_type = -1, bool finish = true,
-                                 bool shares_gpu = false) {
+                                 bool shares_gpu = false, bool follows_compression = false) {
   // lengths are already those after compaction
   LayerState& ls = c->layers[layer];
   hack_step_info_t p{};
@@ -723,7 +723,8 @@ static hack_status_t attend_impl(hack_cache* c, int layer, int scale, const void
       served = only_type == 1 ? n_ctx : bh - n_ctx;
       a.head_order = c->head_order + ((size_t)layer * 2 + only_type) * bh;
     }
-    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, k_new, v_new, served, shares_gpu, st);
+    n = hack::launch_attend_tc(a, a.k_map, a.v_map, a.head_order, q, out, nullptr, k_new, v_new, served, shares_gpu, st,
+                               follows_compression);
   } else {
     n = hack::launch_attend(a, c->cfg.dtype, q, out, st);
   }
@@ -843,7 +844,7 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
       c->launches += n;
       advance_after_compact(c, layer, p);
       s = attend_impl(c, layer, scale, q, out, nullptr, c->side_stream, k, v, seg_new, 1 - trig_type, false, true);
-      if (s == HACK_OK) s = attend_impl(c, layer, scale, q, out, nullptr, st, k, v, seg_new, trig_type, true);
+      if (s == HACK_OK) s = attend_impl(c, layer, scale, q, out, nullptr, st, k, v, seg_new, trig_type, true, false, true);
     }
     // the side stream always comes back to the caller's stream (it may be part of a capture)
     cudaEventRecord(c->ev_join, c->side_stream);
@@ -875,7 +876,8 @@ hack_status_t hack_scale_step(hack_cache_t* c, int32_t layer, int32_t scale, con
   }
   c->launches += n;
   advance_after_compact(c, layer, p);
-  s = attend_impl(c, layer, scale, q, out, nullptr, st, k, v, fused_append ? seg_new : nullptr);
+  s = attend_impl(c, layer, scale, q, out, nullptr, st, k, v, fused_append ? seg_new : nullptr, -1, true, false,
+                  fused_append && compressed);
   if (s == HACK_ERR_CUDA) c->poisoned = true;     // compacted, attention not enqueued
   return s;
 }

@@ -101,10 +101,12 @@ int launch_attend_simt(const StepArgs& a, int dtype, const void* q, void* out, c
 // over [kept - N_k cache rows ; the N_k new rows read from k_new / v_new] and the kernel appends
 // those rows to the cache, so no append or copy launch precedes it for them.  n_heads_served: 0 for
 // every head, else only the first n_heads_served heads of head_order are served (the heads of one type);
-// shares_gpu: another kernel of the step runs beside this launch.
+// shares_gpu: another kernel of the step runs beside this launch.  follows_compression: the launch ahead
+// of this one in the stream is the step's compression launch (the queries, which no kernel of the step
+// writes, may then be read before the dependency wait).
 int launch_attend_tc(const StepArgs& a, const void* k_map, const void* v_map, const int32_t* head_order,
                      const void* q, void* out, float* row_stats, const void* k_new, const void* v_new,
-                     int n_heads_served, bool shares_gpu, cudaStream_t st);
+                     int n_heads_served, bool shares_gpu, cudaStream_t st, bool follows_compression = false);
 constexpr long long kDefaultWaitCycles = 2000000000ll;   // about one second: no wait is legitimately longer
 // Attention variance per (batch, head) over the compacted cache (Eq. 6) from the row statistics of
 // launch_attend_tc; block_var: device scratch [b*H, max_blocks]; sigma: device [b*H].  bf16 only.

@@ -229,3 +229,53 @@ def test_kept_list_beyond_65536_entries():
             d = float(np.max(np.abs(out[0, h].to(torch.float64).cpu().numpy() - o_ref[0, h])))
             assert d <= OUT_TOL["bf16"], f"head {h}: attention output off by {d:.3e}"
     cache.close()
+
+
+@pytest.mark.parametrize("head_dim", [64, 128])
+def test_output_store_stops_at_the_last_query_row(head_dim):
+    """The tensor-core attention writes a 128-row output tile with one tiled store per 64 columns;
+    the scales here have 36, 144 and 400 queries, so the last tile of every head reaches past the
+    head's rows.  The output tensor of every step is a view into a larger buffer that carries a
+    pattern behind it: the pattern has to survive, every head's rows have to be written (no row
+    keeps the fill value), and a second run into a fresh buffer has to give the same bytes (a tile
+    that reached into the next head's rows would race with that head's own store)."""
+    import torch
+    from workloads import SyntheticQKV
+    import paper_2504_09261_b200 as hb
+    cfg = _custom(3, n_heads=3, batch=2, head_dim=head_dim, sides=(1, 2, 6, 12, 20))
+    dev = torch.device("cuda:0")
+    gen = SyntheticQKV(cfg, device=dev)
+    mask = gen.head_is_contextual
+    K = cfg.n_scales
+    qkv = [gen.qkv(0, k) for k in range(K)]
+    guard = 4096                                   # elements behind the output
+    fill = -12345.0                                # rounds to -12352 in bf16; the checks compare raw bits
+
+    def run():
+        cache = hb.HackCache(1, cfg.n_heads, cfg.head_dim, cfg.batch, cfg.sides, hb.HACK_BF16, mask.numpy(), 150, 450,
+                             device=0)
+        bufs, outs = [], []
+        for k in range(K):
+            n = qkv[k][0].numel()
+            buf = torch.full((n + guard,), fill, dtype=torch.bfloat16, device=dev)
+            bufs.append(buf)
+            outs.append(buf[:n].view(qkv[k][0].shape))
+        for k in range(K):
+            q, kk, v = qkv[k]
+            cache.hack_scale_step(0, k, q, kk, v, outs[k])
+        torch.cuda.synchronize()
+        cache.hack_poll_status()                   # raises on a device-side error
+        cache.close()
+        return bufs, outs
+
+    bufs_a, outs_a = run()
+    bufs_b, outs_b = run()
+    fill_bits = torch.tensor([fill], dtype=torch.bfloat16).view(torch.int16).item()
+    for k in range(K):
+        n = qkv[k][0].numel()
+        tail = bufs_a[k][n:].view(torch.int16)
+        assert bool((tail == fill_bits).all()), f"scale {k}: the store wrote behind the output"
+        rows = outs_a[k].reshape(-1, cfg.head_dim).view(torch.int16)
+        untouched = (rows == fill_bits).all(dim=1)
+        assert not bool(untouched.any()), f"scale {k}: {int(untouched.sum())} output rows were never written"
+        assert torch.equal(outs_a[k].view(torch.int16), outs_b[k].view(torch.int16)), f"scale {k}: two runs differ"

@@ -858,6 +858,12 @@ int launch_t(const StepArgs& a, const CUtensorMap& tm_cache, const CUtensorMap& 
     if (ck_active_clusters<D>(a, p) < n_clusters) break;
     cl *= 2;
   }
+  // beside another launch the SMs left over need not hold a power of two per head
+  while (beside && cl < kMaxCluster && (max_chunks + cl) / (cl + 1) >= 2 && n_clusters * (cl + 1) + reserved_sms <= sms) {
+    shape(cl + 1);
+    if (ck_active_clusters<D>(a, p) < n_clusters) break;
+    ++cl;
+  }
   shape(cl);
   if (ck_smem_bytes<D>(p) > kSmemBudget) {
     set_error("compression: shared memory plan beyond the limit");
